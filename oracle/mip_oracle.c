@@ -1,0 +1,150 @@
+/*
+ * CPU oracle for mixed-precision integer (MIP) GEMM and convolution.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, obviously-correct
+ * statement of what the GPU library must compute.  It shares no code, header,
+ * table or helper with the CUDA path and must never be linked into, imported
+ * by or called from the product library; only the test-suite, the smoke check
+ * and the benchmark's cpu-baseline / reference legs use it.
+ *
+ * What is computed (paper, Section 5 opening: INT8 products accumulated in
+ * INT32; Section 7.3: C^q = A^q * B^q; Figure 1: the macro-kernel computes
+ * C += A * B):
+ *
+ *   R(i,j) = (accumulate ? C_in(i,j) : 0) + sum_{k<K} a(i,k) * b(k,j)
+ *
+ * evaluated in 64-bit integers, a(i,k) sign-extended (int8) or zero-extended
+ * (uint8), b(k,j) sign-extended, and then required to fit int32.  A cell whose
+ * exact value does not fit is counted as an overflow cell (the result there is
+ * the low 32 bits, and callers treat the configuration as invalid).
+ *
+ * Layouts: A row-major M x K (a(i,k) = A[i*lda + k]); B column-major K x N
+ * (b(k,j) = B[j*ldb + k]); C row-major M x N (C[i*ldc + j]).  Padding columns
+ * of C (j >= N) are never touched.
+ *
+ * Convolution (paper, Section 7.2, O = Conv(F, I)): direct seven-loop form on
+ * channel-last tensors, never via im2col, so that it shares no structure with
+ * the GPU's lowering:
+ *
+ *   Y[n][ho][wo][co] = sum_{r,s,c} X[n][ho*sh - ph + r*dh][wo*sw - pw + s*dw][c]
+ *                                  * W[co][r][s][c]
+ *
+ * where a term whose input row or column falls outside the image contributes 0.
+ *
+ * Pins: tests/test_oracle_pins.py (brute force on tiny inputs, closed forms,
+ * extremes, range check, checksum identities, NumPy integer matmul, conv vs
+ * explicit im2col, shifted-copy filters).
+ */
+#include <stdint.h>
+#include <stddef.h>
+
+static inline int64_t widen_a(const void *A, int64_t idx, int a_unsigned)
+{
+    if (a_unsigned)
+        return (int64_t)((const uint8_t *)A)[idx];
+    return (int64_t)((const int8_t *)A)[idx];
+}
+
+/*
+ * Returns the number of overflow cells (0 = every cell fits int32), or -1 on
+ * invalid arguments.
+ */
+int64_t mip_oracle_gemm(int a_unsigned, int64_t M, int64_t N, int64_t K,
+                        const void *A, int64_t lda,
+                        const int8_t *B, int64_t ldb,
+                        int32_t *C, int64_t ldc, int accumulate)
+{
+    if (M < 0 || N < 0 || K < 0)
+        return -1;
+    if (M == 0 || N == 0)
+        return 0;
+    if (lda < K || ldb < K || ldc < N)
+        return -1;
+    if (!C || (K > 0 && (!A || !B)))
+        return -1;
+
+    int64_t overflow_cells = 0;
+#pragma omp parallel for schedule(static) reduction(+ : overflow_cells)
+    for (int64_t i = 0; i < M; ++i) {
+        for (int64_t j = 0; j < N; ++j) {
+            int64_t S = 0;
+            for (int64_t k = 0; k < K; ++k) {
+                int64_t a = widen_a(A, i * lda + k, a_unsigned);
+                int64_t b = (int64_t)B[j * ldb + k];
+                S += a * b;
+            }
+            int64_t R = (accumulate ? (int64_t)C[i * ldc + j] : 0) + S;
+            if (R < (int64_t)INT32_MIN || R > (int64_t)INT32_MAX)
+                overflow_cells += 1;
+            C[i * ldc + j] = (int32_t)(uint32_t)(uint64_t)R;
+        }
+    }
+    return overflow_cells;
+}
+
+/*
+ * Direct convolution, uint8 activations (zero-extended) x int8 filters
+ * (sign-extended) -> int32.  X: [Nb][H][W][Cin]; Wt: [Cout][R][S][Cin];
+ * Y: [Nb][Ho][Wo][Cout] with Ho = (H + 2*ph - dh*(R-1) - 1)/sh + 1 (same in w).
+ * Returns overflow-cell count, or -1 on invalid arguments.
+ */
+int64_t mip_oracle_conv(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout,
+                        int64_t R, int64_t S,
+                        int64_t sh, int64_t sw, int64_t ph, int64_t pw,
+                        int64_t dh, int64_t dw,
+                        const uint8_t *X, const int8_t *Wt, int32_t *Y, int accumulate)
+{
+    if (Nb < 0 || H <= 0 || W <= 0 || Cin <= 0 || Cout < 0 || R <= 0 || S <= 0)
+        return -1;
+    if (sh <= 0 || sw <= 0 || dh <= 0 || dw <= 0 || ph < 0 || pw < 0)
+        return -1;
+    int64_t eh = H + 2 * ph - dh * (R - 1) - 1;
+    int64_t ew = W + 2 * pw - dw * (S - 1) - 1;
+    if (eh < 0 || ew < 0)
+        return -1;
+    int64_t Ho = eh / sh + 1;
+    int64_t Wo = ew / sw + 1;
+    if (Nb == 0 || Cout == 0)
+        return 0;
+    if (!X || !Wt || !Y)
+        return -1;
+
+    int64_t overflow_cells = 0;
+#pragma omp parallel for collapse(2) schedule(static) reduction(+ : overflow_cells)
+    for (int64_t n = 0; n < Nb; ++n) {
+        for (int64_t ho = 0; ho < Ho; ++ho) {
+            for (int64_t wo = 0; wo < Wo; ++wo) {
+                for (int64_t co = 0; co < Cout; ++co) {
+                    int64_t acc = 0;
+                    for (int64_t r = 0; r < R; ++r) {
+                        int64_t h = ho * sh - ph + r * dh;
+                        if (h < 0 || h >= H)
+                            continue;
+                        for (int64_t s = 0; s < S; ++s) {
+                            int64_t w = wo * sw - pw + s * dw;
+                            if (w < 0 || w >= W)
+                                continue;
+                            const uint8_t *x = X + ((n * H + h) * W + w) * Cin;
+                            const int8_t *f = Wt + ((co * R + r) * S + s) * Cin;
+                            for (int64_t c = 0; c < Cin; ++c)
+                                acc += (int64_t)x[c] * (int64_t)f[c];
+                        }
+                    }
+                    int64_t yi = ((n * Ho + ho) * Wo + wo) * Cout + co;
+                    int64_t Rv = (accumulate ? (int64_t)Y[yi] : 0) + acc;
+                    if (Rv < (int64_t)INT32_MIN || Rv > (int64_t)INT32_MAX)
+                        overflow_cells += 1;
+                    Y[yi] = (int32_t)(uint32_t)(uint64_t)Rv;
+                }
+            }
+        }
+    }
+    return overflow_cells;
+}
+
+#ifdef _OPENMP
+#include <omp.h>
+int mip_oracle_threads(void) { return omp_get_max_threads(); }
+#else
+int mip_oracle_threads(void) { return 1; }
+#endif

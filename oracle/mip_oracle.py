@@ -1,0 +1,144 @@
+"""ctypes front end of the CPU oracle (``mip_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: nothing in the product package may import this
+module.  It compiles the plain-C oracle with gcc on first use (OpenMP over
+output rows) and exposes it on NumPy arrays.  The arithmetic lives in the C
+file; this module only marshals arguments.
+
+Definitions followed: exact INT8 x INT8 -> INT32 GEMM (paper Section 5
+opening, Section 7.3, Figure 1) and the convolution operator of Section 7.2.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "mip_oracle.c")
+_LIB = os.path.join(_HERE, "libmip_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle shared object next to its source; returns its path."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + ".tmp.%d" % os.getpid()
+            cmd = ["gcc", "-O3", "-march=native", "-fopenmp", "-fPIC", "-shared",
+                   "-std=c11", "-Wall", "-Wextra", "-o", tmp, _SRC]
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        i64, vp, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+        lib.mip_oracle_gemm.restype = i64
+        lib.mip_oracle_gemm.argtypes = [ci, i64, i64, i64, vp, i64, vp, i64, vp, i64, ci]
+        lib.mip_oracle_conv.restype = i64
+        lib.mip_oracle_conv.argtypes = [i64] * 13 + [vp, vp, vp, ci]
+        lib.mip_oracle_threads.restype = ci
+        lib.mip_oracle_threads.argtypes = []
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    """Number of OpenMP threads the oracle will use."""
+    return int(_load().mip_oracle_threads())
+
+
+class OracleOverflow(ArithmeticError):
+    """The exact result of some cell does not fit int32."""
+
+
+def _ptr(a: np.ndarray) -> int:
+    return a.ctypes.data
+
+
+def gemm(A: np.ndarray, B: np.ndarray, M: int, N: int, K: int, *, lda: int | None = None,
+         ldb: int | None = None, C: np.ndarray | None = None, ldc: int | None = None,
+         accumulate: bool = False, allow_overflow: bool = False) -> np.ndarray:
+    """C = [C +] A * B, exact.
+
+    ``A``: flat or 2-D C-contiguous buffer of int8 (signed mode) or uint8
+    (unsigned mode), row-major M x K with pitch ``lda``.  ``B``: int8 buffer,
+    column-major K x N, i.e. N runs of K bytes with pitch ``ldb``.  ``C``:
+    int32 buffer with pitch ``ldc`` (allocated, zero-filled, when omitted); it is
+    updated in place and returned.  Raises :class:`OracleOverflow` if any exact
+    value leaves the int32 range, unless ``allow_overflow``.
+    """
+    if A.dtype == np.int8:
+        a_unsigned = 0
+    elif A.dtype == np.uint8:
+        a_unsigned = 1
+    else:
+        raise TypeError("A must be int8 or uint8")
+    if B.dtype != np.int8:
+        raise TypeError("B must be int8")
+    lda = K if lda is None else lda
+    ldb = K if ldb is None else ldb
+    ldc = N if ldc is None else ldc
+    if C is None:
+        C = np.zeros(max(M, 0) * ldc, dtype=np.int32)
+    if C.dtype != np.int32:
+        raise TypeError("C must be int32")
+    for arr in (A, B, C):
+        if not arr.flags["C_CONTIGUOUS"]:
+            raise ValueError("buffers must be C-contiguous")
+    if M > 0 and N > 0:
+        if K > 0 and (A.size < (M - 1) * lda + K or B.size < (N - 1) * ldb + K):
+            raise ValueError("A or B buffer too small for the stated pitch")
+        if C.size < (M - 1) * ldc + N:
+            raise ValueError("C buffer too small for the stated pitch")
+    rc = _load().mip_oracle_gemm(a_unsigned, M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                 1 if accumulate else 0)
+    if rc < 0:
+        raise ValueError("mip_oracle_gemm rejected its arguments")
+    if rc > 0 and not allow_overflow:
+        raise OracleOverflow("%d cells do not fit int32" % rc)
+    return C
+
+
+def conv_out_hw(H, W, R, S, stride, pad, dil):
+    """Output extent of the convolution (paper Section 7.2 shapes)."""
+    Ho = (H + 2 * pad[0] - dil[0] * (R - 1) - 1) // stride[0] + 1
+    Wo = (W + 2 * pad[1] - dil[1] * (S - 1) - 1) // stride[1] + 1
+    return Ho, Wo
+
+
+def conv(X: np.ndarray, Wt: np.ndarray, *, stride=(1, 1), pad=(0, 0), dil=(1, 1),
+         Y: np.ndarray | None = None, accumulate: bool = False,
+         allow_overflow: bool = False) -> np.ndarray:
+    """Y = [Y +] Conv(Wt, X): X uint8 [Nb][H][W][Cin], Wt int8 [Cout][R][S][Cin],
+    Y int32 [Nb][Ho][Wo][Cout]; out-of-image taps contribute zero."""
+    if X.dtype != np.uint8 or Wt.dtype != np.int8:
+        raise TypeError("X must be uint8 and Wt int8")
+    Nb, H, W, Cin = X.shape
+    Cout, R, S, Cin2 = Wt.shape
+    if Cin != Cin2:
+        raise ValueError("channel mismatch")
+    Ho, Wo = conv_out_hw(H, W, R, S, stride, pad, dil)
+    X = np.ascontiguousarray(X)
+    Wt = np.ascontiguousarray(Wt)
+    if Y is None:
+        Y = np.zeros((Nb, Ho, Wo, Cout), dtype=np.int32)
+    if Y.dtype != np.int32 or Y.shape != (Nb, Ho, Wo, Cout) or not Y.flags["C_CONTIGUOUS"]:
+        raise ValueError("Y must be a contiguous int32 [Nb][Ho][Wo][Cout] array")
+    rc = _load().mip_oracle_conv(Nb, H, W, Cin, Cout, R, S, stride[0], stride[1], pad[0], pad[1],
+                                 dil[0], dil[1], _ptr(X), _ptr(Wt), _ptr(Y), 1 if accumulate else 0)
+    if rc < 0:
+        raise ValueError("mip_oracle_conv rejected its arguments")
+    if rc > 0 and not allow_overflow:
+        raise OracleOverflow("%d cells do not fit int32" % rc)
+    return Y
