@@ -1,0 +1,178 @@
+/*
+ * libmipgemm -- exact mixed-precision integer GEMM for NVIDIA B200 (sm_100a).
+ *
+ *     C(int32) [+]= A(int8 | uint8) * B(int8)
+ *
+ * This is the hot path of "mixed-precision integer (MIP) GEMM" for quantized
+ * inference: 8-bit operands, 32-bit exact accumulation (paper Section 5,
+ * opening paragraphs; Section 7.3, C^q = A^q B^q; Figure 1, C += A B), its use
+ * for convolution through the im2col lowering (Section 7.2) and for the
+ * weight-by-activation GEMMs of a transformer encoder (Table 5), and the
+ * matrix-vector / skinny case of the final fully connected layer (Section 7.4,
+ * "2mn useful operations").
+ *
+ * Conventions common to every entry point
+ * ---------------------------------------
+ *  - All data pointers are DEVICE pointers on the current CUDA device, owned by
+ *    the caller; the library neither frees nor retains them.  `stream` is a
+ *    cudaStream_t passed as void* (NULL = legacy default stream).  Calls are
+ *    asynchronous: they return after the work has been enqueued.
+ *  - Return value: MIPGEMM_OK (0) or one of the error codes below.  Argument
+ *    errors are detected synchronously and nothing is enqueued.  Device-side
+ *    problems (a bounded wait that ran out) are reported by
+ *    mipgemm_device_status().
+ *  - Exactness: the result equals the mathematical value whenever that value
+ *    fits int32.  With accumulate == 0 this is unconditional, because K is
+ *    limited so that the worst case cannot overflow: K <= 131071 in s8*s8 mode
+ *    (128*128*K <= 2^31-1) and K <= 65793 in u8*s8 mode (255*128*K <= 2^31);
+ *    larger K returns MIPGEMM_ERR_K_TOO_LARGE.  With accumulate != 0 the sum
+ *    C_in + A*B wraps modulo 2^32 if it leaves the int32 range; keeping it in
+ *    range is the caller's responsibility.  There is no saturation anywhere.
+ *  - A, B and C must not overlap.  A and B need byte alignment only; C needs
+ *    4-byte alignment.  Any pitch >= the minimum is accepted; operands whose
+ *    base or pitch is not 16-byte aligned are first copied into scratch memory
+ *    (see "Scratch memory").
+ *  - Padding elements of C (columns N .. ldc-1 of a row) are never written.
+ *  - M == 0 or N == 0: no-op, MIPGEMM_OK.  K == 0: C is zero-filled
+ *    (accumulate == 0) or left unchanged (accumulate != 0).
+ *
+ * Scratch memory
+ * --------------
+ * Some calls need global scratch memory (operand re-pitching, the explicit
+ * im2col matrix for convolutions the tensor-memory-accelerator cannot gather,
+ * split-K partial sums).  By default it is taken with cudaMallocAsync on the
+ * call's stream and released with cudaFreeAsync after the last kernel of the
+ * call.  A caller may instead lend a buffer with mipgemm_set_workspace(); calls
+ * that need more than was lent fail with MIPGEMM_ERR_WORKSPACE.  A lent buffer
+ * is shared by all calls: calls that use it must be ordered on one stream.
+ */
+#ifndef MIPGEMM_H_
+#define MIPGEMM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MIPGEMM_OK = 0,
+    MIPGEMM_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, pitch too small, bad conv geometry */
+    MIPGEMM_ERR_K_TOO_LARGE = 2, /* exactness could not be guaranteed (see above)                  */
+    MIPGEMM_ERR_UNSUPPORTED = 3, /* current device is not compute capability 10.0                  */
+    MIPGEMM_ERR_WORKSPACE = 4,   /* scratch memory could not be obtained / lent buffer too small   */
+    MIPGEMM_ERR_CUDA = 5,        /* a CUDA call failed; see mipgemm_last_cuda_error()              */
+    MIPGEMM_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (kernel returned early)     */
+} mipgemm_status_t;
+
+/* Which kernel family served the most recent GEMM/conv call of this thread (test hook). */
+typedef enum {
+    MIPGEMM_PATH_NONE = 0,
+    MIPGEMM_PATH_DENSE = 1,       /* TMA + tcgen05.mma.kind::i8, one CTA per tile            */
+    MIPGEMM_PATH_DENSE_PAIR = 2,  /* same, CTA pairs (cta_group::2)                          */
+    MIPGEMM_PATH_SKINNY = 3,      /* M <= 16 streaming kernel                                */
+    MIPGEMM_PATH_TRIVIAL = 4,     /* K == 0 fill or empty problem                            */
+    MIPGEMM_PATH_REPACK = 0x100,  /* flag: an operand was re-pitched into scratch first      */
+    MIPGEMM_PATH_SPLITK = 0x200,  /* flag: K was split and reduced with integer atomics      */
+    MIPGEMM_PATH_IM2COL_TMA = 0x400,   /* flag: conv gathered by TMA im2col loads            */
+    MIPGEMM_PATH_IM2COL_EXPLICIT = 0x800 /* flag: conv materialised the augmented matrix     */
+} mipgemm_path_t;
+
+/*
+ * C = [C +] A * B, signed 8-bit A.   (Paper: Figure 1 and Section 5 -- INT8
+ * products, INT32 accumulation; the result is the exact integer matrix product.)
+ *
+ *   A : row-major    M x K, a(i,k) = A[i*lda + k], lda >= K          (device, read)
+ *   B : column-major K x N, b(k,j) = B[j*ldb + k], ldb >= K          (device, read)
+ *       -- i.e. N runs of K contiguous bytes, the usual [out][in] weight layout
+ *   C : row-major    M x N, c(i,j) = C[i*ldc + j], ldc >= N          (device, read/write)
+ *   accumulate : 0 -> C = A*B, previous contents of C are ignored;
+ *                nonzero -> C += A*B.
+ *   stream : cudaStream_t.
+ */
+int mipgemm_s8s8s32(int64_t M, int64_t N, int64_t K,
+                    const int8_t *A, int64_t lda,
+                    const int8_t *B, int64_t ldb,
+                    int32_t *C, int64_t ldc,
+                    int accumulate, void *stream);
+
+/* Same with unsigned 8-bit A (zero-extended), e.g. post-ReLU activations.  The
+ * paper's kernels are signed*signed; the unsigned variant follows the same
+ * definition with a(i,k) in [0,255] and has no zero-point term. */
+int mipgemm_u8s8s32(int64_t M, int64_t N, int64_t K,
+                    const uint8_t *A, int64_t lda,
+                    const int8_t *B, int64_t ldb,
+                    int32_t *C, int64_t ldc,
+                    int accumulate, void *stream);
+
+/*
+ * Y = [Y +] Conv(Wt, X): channel-last convolution lowered to the GEMM above
+ * (paper Section 7.2: O = Conv(F, I), im2col lowering, the cost of the
+ * lowering is part of the operator).  GEMM view: M = Nb*Ho*Wo output pixels,
+ * N = Cout, K = R*S*Cin ordered (r, s, c).
+ *
+ *   X  : [Nb][H][W][Cin]      uint8, dense                           (device, read)
+ *   Wt : [Cout][R][S][Cin]    int8, dense                            (device, read)
+ *   Y  : [Nb][Ho][Wo][Cout]   int32, dense                           (device, read/write)
+ *        Ho = (H + 2*pad_h - dil_h*(R-1) - 1)/stride_h + 1, Wo likewise.
+ *   Taps that fall outside the image contribute 0 (scale-only quantization, no
+ *   zero point).  K = R*S*Cin obeys the u8*s8 limit above.
+ */
+int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout,
+                         int R, int S, int stride_h, int stride_w,
+                         int pad_h, int pad_w, int dil_h, int dil_w,
+                         const uint8_t *X, const int8_t *Wt, int32_t *Y,
+                         int accumulate, void *stream);
+
+/* ---- support calls (no counterpart in the paper) ---- */
+
+/* Synchronises `stream` and returns MIPGEMM_OK, MIPGEMM_ERR_TIMEOUT if any kernel
+ * since the last call gave up a bounded wait (the flag is then cleared), or
+ * MIPGEMM_ERR_CUDA if the synchronisation itself failed. */
+int mipgemm_device_status(void *stream);
+
+/* Lend (dev_ptr != NULL, 256-byte aligned) or withdraw (dev_ptr == NULL) a scratch
+ * buffer for the current device. */
+int mipgemm_set_workspace(void *dev_ptr, size_t bytes);
+
+/* Scratch bytes the corresponding call would need (0 = none). `a_unsigned` selects
+ * the u8 variant.  Pointers matter only through their alignment. */
+size_t mipgemm_workspace_query_gemm(int64_t M, int64_t N, int64_t K,
+                                    const void *A, int64_t lda,
+                                    const void *B, int64_t ldb,
+                                    const void *C, int64_t ldc, int accumulate);
+size_t mipgemm_workspace_query_conv(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout,
+                                    int R, int S, int stride_h, int stride_w,
+                                    int pad_h, int pad_w, int dil_h, int dil_w);
+
+/* Path taken by this thread's most recent call: a mipgemm_path_t value or-ed with flags. */
+int mipgemm_last_path(void);
+
+/* cudaError_t of the most recent failing CUDA call of this thread (0 = none). */
+int mipgemm_last_cuda_error(void);
+
+const char *mipgemm_status_string(int status);
+
+/* major*10000 + minor*100 + patch */
+int mipgemm_version(void);
+
+/*
+ * Tensor-pipe peak probe (the analogue of the paper's Table 1 instruction-rate
+ * micro-benchmarks): every SM issues `iters` groups of tcgen05.mma.kind::i8
+ * (M=128, N=256, K=32 per instruction, 4 per group) on operands resident in
+ * shared memory, nothing is loaded from or stored to global memory except one
+ * word per CTA.  On return *ops_per_launch = 2*128*256*128*iters*CTAs.  The
+ * caller times the launch.  `sink` : device, >= 4*grid bytes.
+ */
+int mipgemm_probe_i8_peak(int iters, int *grid_out, double *ops_per_launch,
+                          int32_t *sink, void *stream);
+
+/* Overrides for experiments: tile width (0 = heuristic; 64, 128 or 256), pipeline
+ * depth (0 = heuristic), split-K factor (0 = heuristic, 1 = off), force path. */
+int mipgemm_set_tuning(int block_n, int stages, int split_k, int force_path);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MIPGEMM_H_ */

@@ -1,0 +1,148 @@
+"""Thin ctypes binding of ``libmipgemm.so``: same names as ``include/mipgemm.h``.
+
+Argument marshalling only -- every step of the method runs in the CUDA kernels
+behind the C ABI.  Tensors are ``torch`` CUDA tensors (or raw device addresses as
+``int``); PyTorch is used for device memory and streams, nothing else.  There is
+no CPU fallback: if the shared library has not been built, importing this module
+raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmipgemm.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "libmipgemm.so is missing (%s). Build it with `python -m paper_2506_11728_b200.build` "
+        "or `__graft_entry__.build()`; there is no fallback path." % LIB_PATH)
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+_i64, _int, _vp, _sz = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t
+
+OK, ERR_INVALID_ARG, ERR_K_TOO_LARGE, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
+PATH_NONE, PATH_DENSE, PATH_DENSE_PAIR, PATH_SKINNY, PATH_TRIVIAL = range(5)
+PATH_MASK = 0xFF
+PATH_REPACK, PATH_SPLITK, PATH_IM2COL_TMA, PATH_IM2COL_EXPLICIT = 0x100, 0x200, 0x400, 0x800
+
+#: every symbol include/mipgemm.h declares, with (restype, argtypes)
+SIGNATURES = {
+    "mipgemm_s8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
+    "mipgemm_u8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
+    "mipgemm_conv_u8s8s32": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, _int, _vp]),
+    "mipgemm_device_status": (_int, [_vp]),
+    "mipgemm_set_workspace": (_int, [_vp, _sz]),
+    "mipgemm_workspace_query_gemm": (_sz, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int]),
+    "mipgemm_workspace_query_conv": (_sz, [_i64] * 5 + [_int] * 8),
+    "mipgemm_last_path": (_int, []),
+    "mipgemm_last_cuda_error": (_int, []),
+    "mipgemm_status_string": (ctypes.c_char_p, [_int]),
+    "mipgemm_version": (_int, []),
+    "mipgemm_probe_i8_peak": (_int, [_int, ctypes.POINTER(_int), ctypes.POINTER(ctypes.c_double), _vp, _vp]),
+    "mipgemm_set_tuning": (_int, [_int, _int, _int, _int]),
+}
+for _name, (_res, _args) in SIGNATURES.items():
+    _fn = getattr(_lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+
+class MipGemmError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        super().__init__("libmipgemm: %s (status %d, cuda error %d)" % (
+            mipgemm_status_string(status), status, mipgemm_last_cuda_error()))
+
+
+def _ptr(x) -> int:
+    if x is None:
+        return 0
+    if isinstance(x, int):
+        return x
+    return x.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(status: int, check: bool) -> int:
+    if check and status != OK:
+        raise MipGemmError(status)
+    return status
+
+
+def mipgemm_s8s8s32(M, N, K, A, lda, B, ldb, C, ldc, accumulate=0, stream=None, check=True) -> int:
+    """C[int32, MxN, pitch ldc] (+)= A[int8, MxK row-major, pitch lda] * B[int8, KxN column-major, pitch ldb]."""
+    return _check(_lib.mipgemm_s8s8s32(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                       int(bool(accumulate)), _stream(stream)), check)
+
+
+def mipgemm_u8s8s32(M, N, K, A, lda, B, ldb, C, ldc, accumulate=0, stream=None, check=True) -> int:
+    """Same with unsigned 8-bit A."""
+    return _check(_lib.mipgemm_u8s8s32(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                       int(bool(accumulate)), _stream(stream)), check)
+
+
+def mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w,
+                         X, Wt, Y, accumulate=0, stream=None, check=True) -> int:
+    """Y[int32 NHWC] (+)= Conv(Wt[int8 KRSC], X[uint8 NHWC])."""
+    return _check(_lib.mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
+                                            dil_h, dil_w, _ptr(X), _ptr(Wt), _ptr(Y),
+                                            int(bool(accumulate)), _stream(stream)), check)
+
+
+def mipgemm_device_status(stream=None) -> int:
+    return _lib.mipgemm_device_status(_stream(stream))
+
+
+def mipgemm_set_workspace(buf, nbytes: int = 0) -> int:
+    return _lib.mipgemm_set_workspace(_ptr(buf), nbytes)
+
+
+def mipgemm_workspace_query_gemm(M, N, K, A, lda, B, ldb, C, ldc, accumulate=0) -> int:
+    return _lib.mipgemm_workspace_query_gemm(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                             int(bool(accumulate)))
+
+
+def mipgemm_workspace_query_conv(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
+                                 dil_h, dil_w) -> int:
+    return _lib.mipgemm_workspace_query_conv(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
+                                             dil_h, dil_w)
+
+
+def mipgemm_last_path() -> int:
+    return _lib.mipgemm_last_path()
+
+
+def mipgemm_last_cuda_error() -> int:
+    return _lib.mipgemm_last_cuda_error()
+
+
+def mipgemm_status_string(status: int) -> str:
+    return _lib.mipgemm_status_string(status).decode()
+
+
+def mipgemm_version() -> int:
+    return _lib.mipgemm_version()
+
+
+def mipgemm_probe_i8_peak(iters: int, sink, stream=None):
+    """Launches the tensor-pipe probe; returns (grid, ops_per_launch)."""
+    grid = _int(0)
+    ops = ctypes.c_double(0.0)
+    st = _lib.mipgemm_probe_i8_peak(iters, ctypes.byref(grid), ctypes.byref(ops), _ptr(sink), _stream(stream))
+    _check(st, True)
+    return grid.value, ops.value
+
+
+def mipgemm_set_tuning(block_n=0, stages=0, split_k=0, force_path=0) -> int:
+    return _check(_lib.mipgemm_set_tuning(block_n, stages, split_k, force_path), True)

@@ -1,0 +1,564 @@
+// C-ABI entry points of libmipgemm: argument validation, path selection, tensor-map
+// construction, scratch-memory handling and kernel launches.  No arithmetic of the
+// method happens on the host.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/mipgemm.h"
+#include "internal.h"
+
+namespace {
+
+using namespace mip;
+
+thread_local int tl_last_path = MIPGEMM_PATH_NONE;
+thread_local int tl_last_cuda_error = 0;
+
+struct Tuning {
+    int block_n = 0, stages = 0, split_k = 0, force_path = 0;
+};
+Tuning g_tuning;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr int kMaxDevices = 64;
+struct DeviceState {
+    bool ready = false;
+    int status = MIPGEMM_OK;
+    int sm_count = 0;
+    unsigned int* status_word = nullptr;   // device
+    void* lent = nullptr;
+    size_t lent_bytes = 0;
+};
+DeviceState g_dev[kMaxDevices];
+std::mutex g_mutex;
+EncodeTiledFn g_encode_tiled = nullptr;
+EncodeIm2colFn g_encode_im2col = nullptr;
+
+int cuda_fail(cudaError_t e) {
+    tl_last_cuda_error = static_cast<int>(e);
+    return MIPGEMM_ERR_CUDA;
+}
+
+// Once per device: capability check, driver entry points, kernel attributes, status word.
+int get_device(DeviceState** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return MIPGEMM_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState& d = g_dev[dev];
+    if (!d.ready) {
+        int major = 0, minor = 0;
+        if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return cuda_fail(e);
+        if (major != 10 || minor != 0) {
+            d.status = MIPGEMM_ERR_UNSUPPORTED;
+        } else {
+            if (!g_encode_tiled) {
+                void* fn = nullptr;
+                cudaDriverEntryPointQueryResult qr;
+                e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr);
+                if (e != cudaSuccess || qr != cudaDriverEntryPointSuccess || !fn)
+                    return cuda_fail(e == cudaSuccess ? cudaErrorUnknown : e);
+                g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+                fn = nullptr;
+                e = cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn, cudaEnableDefault, &qr);
+                if (e != cudaSuccess || qr != cudaDriverEntryPointSuccess || !fn)
+                    return cuda_fail(e == cudaSuccess ? cudaErrorUnknown : e);
+                g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(fn);
+            }
+            if ((e = dense_init()) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaMalloc(&d.status_word, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaMemset(d.status_word, 0, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
+            d.status = MIPGEMM_OK;
+        }
+        d.ready = true;
+    }
+    *out = &d;
+    return d.status;
+}
+
+// Scratch memory for one call: a slice of the lent buffer, or a stream-ordered allocation.
+struct Scratch {
+    DeviceState* dev;
+    cudaStream_t stream;
+    void* base = nullptr;
+    size_t size = 0, used = 0;
+    bool owned = false;
+    Scratch(DeviceState* d, cudaStream_t s) : dev(d), stream(s) {}
+    int reserve(size_t bytes) {
+        if (bytes == 0) return MIPGEMM_OK;
+        if (dev->lent) {
+            if (bytes > dev->lent_bytes) return MIPGEMM_ERR_WORKSPACE;
+            base = dev->lent;
+        } else {
+            cudaError_t e = cudaMallocAsync(&base, bytes, stream);
+            if (e != cudaSuccess) {
+                tl_last_cuda_error = static_cast<int>(e);
+                (void)cudaGetLastError();
+                return MIPGEMM_ERR_WORKSPACE;
+            }
+            owned = true;
+        }
+        size = bytes;
+        return MIPGEMM_OK;
+    }
+    void* take(size_t bytes) {
+        void* p = static_cast<char*>(base) + used;
+        used += (bytes + 255) & ~static_cast<size_t>(255);
+        return p;
+    }
+    ~Scratch() {
+        if (owned && base) (void)cudaFreeAsync(base, stream);
+    }
+};
+
+size_t align256(size_t b) { return (b + 255) & ~static_cast<size_t>(255); }
+long long round_up(long long v, long long m) { return (v + m - 1) / m * m; }
+bool aligned16(const void* p, long long pitch) {
+    return reinterpret_cast<uintptr_t>(p) % 16 == 0 && pitch % 16 == 0;
+}
+
+int encode_tiled_2d(CUtensorMap* map, const void* base, long long inner, long long outer, long long pitch,
+                    int box_inner, int box_outer) {
+    cuuint64_t dims[2] = {static_cast<cuuint64_t>(inner), static_cast<cuuint64_t>(outer)};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch)};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(box_inner), static_cast<cuuint32_t>(box_outer)};
+    cuuint32_t estr[2] = {1, 1};
+    const CUtensorMapSwizzle sw = box_inner == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+    CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides,
+                                box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        tl_last_cuda_error = 100000 + static_cast<int>(r);
+        return MIPGEMM_ERR_CUDA;
+    }
+    return MIPGEMM_OK;
+}
+
+struct ConvGeom {
+    long long Nb, H, W, Cin, Cout, Ho, Wo;
+    int R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
+};
+
+int encode_im2col(CUtensorMap* map, const void* X, const ConvGeom& g, int channels_per_pixel,
+                  int pixels_per_column) {
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(g.Cin), static_cast<cuuint64_t>(g.W),
+                          static_cast<cuuint64_t>(g.H), static_cast<cuuint64_t>(g.Nb)};
+    cuuint64_t strides[3] = {static_cast<cuuint64_t>(g.Cin), static_cast<cuuint64_t>(g.W * g.Cin),
+                             static_cast<cuuint64_t>(g.H * g.W * g.Cin)};
+    int lower[2] = {-g.pad_w, -g.pad_h};
+    int upper[2] = {g.pad_w - (g.S - 1) * g.dil_w, g.pad_h - (g.R - 1) * g.dil_h};
+    cuuint32_t estr[4] = {1, static_cast<cuuint32_t>(g.stride_w), static_cast<cuuint32_t>(g.stride_h), 1};
+    const CUtensorMapSwizzle sw =
+        channels_per_pixel == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+    CUresult r = g_encode_im2col(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(X), dims, strides,
+                                 lower, upper, static_cast<cuuint32_t>(channels_per_pixel),
+                                 static_cast<cuuint32_t>(pixels_per_column), estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        tl_last_cuda_error = 100000 + static_cast<int>(r);
+        return MIPGEMM_ERR_CUDA;
+    }
+    return MIPGEMM_OK;
+}
+
+uint32_t pow2_at_least(uint32_t v) {
+    uint32_t p = 32;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+// Tile width, pipeline depth and split-K for an M x N x K problem (k-block = block_k bytes).
+struct Plan {
+    int block_n, stages, split_k, kb_per_split, k_blocks, tiles_m, tiles_n;
+};
+
+Plan make_plan(long long M, long long N, long long K, int block_k, int sm_count) {
+    Plan pl{};
+    pl.tiles_m = static_cast<int>((M + kBlockM - 1) / kBlockM);
+    pl.k_blocks = static_cast<int>((K + block_k - 1) / block_k);
+    auto tiles_for = [&](int bn) { return static_cast<long long>(pl.tiles_m) * ((N + bn - 1) / bn); };
+    int bn;
+    if (g_tuning.block_n) {
+        bn = g_tuning.block_n;
+    } else if (N <= 64) {
+        bn = 64;
+    } else if (N <= 128) {
+        bn = 128;
+    } else if (tiles_for(256) >= sm_count) {
+        bn = 256;
+    } else if (tiles_for(128) >= sm_count || N <= 256 + 128) {
+        bn = 128;
+    } else {
+        bn = 64;
+        if (tiles_for(64) < sm_count) bn = 128;   // too few tiles either way: prefer the wider MMA, split K
+    }
+    pl.block_n = bn;
+    pl.tiles_n = static_cast<int>((N + bn - 1) / bn);
+    const int stage_bytes = kBlockM * block_k + bn * block_k;
+    int stages = (kSmemBudget - kCtrlBytes - 1024) / stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (g_tuning.stages) stages = g_tuning.stages < stages ? g_tuning.stages : stages;
+    if (stages < 2) stages = 2;
+    pl.stages = stages;
+    int split = 1;
+    const long long tiles = static_cast<long long>(pl.tiles_m) * pl.tiles_n;
+    if (g_tuning.split_k) {
+        split = g_tuning.split_k;
+    } else if (tiles * 2 <= sm_count && pl.k_blocks >= 8) {
+        split = static_cast<int>(sm_count / tiles);
+        const int max_split = pl.k_blocks / 4;
+        if (split > max_split) split = max_split;
+    }
+    if (split > pl.k_blocks) split = pl.k_blocks;
+    if (split < 1) split = 1;
+    pl.kb_per_split = (pl.k_blocks + split - 1) / split;
+    pl.split_k = (pl.k_blocks + pl.kb_per_split - 1) / pl.kb_per_split;
+    return pl;
+}
+
+void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32_t* C, long long ldc,
+                 int block_k, bool a_unsigned, int accumulate, DeviceState* dev) {
+    p.C = C;
+    p.ldc = ldc;
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.k_blocks = pl.k_blocks;
+    p.block_n = pl.block_n;
+    p.block_k = block_k;
+    p.stages = pl.stages;
+    p.tiles_m = pl.tiles_m;
+    p.tiles_n = pl.tiles_n;
+    p.split_k = pl.split_k;
+    p.kb_per_split = pl.kb_per_split;
+    p.group_n = 8;
+    p.use_red = pl.split_k > 1 ? 1 : 0;
+    p.accumulate = p.use_red ? 0 : (accumulate ? 1 : 0);
+    const uintptr_t c_addr = reinterpret_cast<uintptr_t>(C);
+    p.store_vec = (c_addr % 32 == 0 && ldc % 8 == 0) ? 8 : ((c_addr % 16 == 0 && ldc % 4 == 0) ? 4 : 1);
+    p.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) |
+              (static_cast<uint32_t>(pl.block_n >> 3) << 17) | (static_cast<uint32_t>(kBlockM >> 4) << 24);
+    p.tmem_cols = pow2_at_least(2u * pl.block_n);
+    p.a_im2col = 0;
+    p.status = dev->status_word;
+    p.wait_budget_ns = 4000000000ull;
+}
+
+int run_dense(DenseParams& p, const Plan& pl, long long M, long long N, int32_t* C, long long ldc,
+              int accumulate, DeviceState* dev, cudaStream_t stream) {
+    if (pl.split_k > 1 && !accumulate) {
+        cudaError_t e = launch_fill_zero(C, ldc, M, N, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    const long long units = static_cast<long long>(pl.tiles_m) * pl.tiles_n * pl.split_k;
+    const int grid = static_cast<int>(units < dev->sm_count ? units : dev->sm_count);
+    const size_t smem = static_cast<size_t>(pl.stages) * (kBlockM * p.block_k + pl.block_n * p.block_k) +
+                        kCtrlBytes + 1024;
+    cudaError_t e = launch_dense(p, grid, smem, stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return MIPGEMM_OK;
+}
+
+size_t gemm_scratch_bytes(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, const void* B,
+                          int64_t ldb) {
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    const long long pitch = round_up(K, 16);
+    size_t need = 0;
+    if (!aligned16(A, lda)) need += align256(static_cast<size_t>(M) * pitch);
+    if (!aligned16(B, ldb)) need += align256(static_cast<size_t>(N) * pitch);
+    return need;
+}
+
+// `outer`: scratch already reserved by the caller (the explicit-im2col convolution), from
+// which this call takes its own share; nullptr = reserve what is needed here.
+int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, const int8_t* B,
+              int64_t ldb, int32_t* C, int64_t ldc, int accumulate, void* stream_v, int path_flags,
+              Scratch* outer = nullptr) {
+    tl_last_path = MIPGEMM_PATH_NONE;
+    if (M < 0 || N < 0 || K < 0) return MIPGEMM_ERR_INVALID_ARG;
+    if (M > 0x7FFFFF00LL || N > 0x7FFFFF00LL) return MIPGEMM_ERR_INVALID_ARG;
+    if (lda < K || ldb < K || ldc < N) return MIPGEMM_ERR_INVALID_ARG;
+    if (K > (a_unsigned ? 65793 : 131071)) return MIPGEMM_ERR_K_TOO_LARGE;
+    if (M == 0 || N == 0) {
+        tl_last_path = MIPGEMM_PATH_TRIVIAL | path_flags;
+        return MIPGEMM_OK;
+    }
+    if (!C || reinterpret_cast<uintptr_t>(C) % 4 != 0) return MIPGEMM_ERR_INVALID_ARG;
+    if (K > 0 && (!A || !B)) return MIPGEMM_ERR_INVALID_ARG;
+    DeviceState* dev = nullptr;
+    int st = get_device(&dev);
+    if (st != MIPGEMM_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+
+    if (K == 0) {
+        tl_last_path = MIPGEMM_PATH_TRIVIAL | path_flags;
+        if (!accumulate) {
+            cudaError_t e = launch_fill_zero(C, ldc, M, N, stream);
+            if (e != cudaSuccess) return cuda_fail(e);
+        }
+        return MIPGEMM_OK;
+    }
+
+    // ---- skinny path
+    if (M <= 16 && g_tuning.force_path != MIPGEMM_PATH_DENSE) {
+        SkinnyParams sp{A, lda, B, ldb, C, ldc, static_cast<int>(M), static_cast<int>(N),
+                        static_cast<int>(K), a_unsigned ? 1 : 0, accumulate ? 1 : 0};
+        if (skinny_supported(sp)) {
+            cudaError_t e = launch_skinny(sp, stream);
+            if (e != cudaSuccess) return cuda_fail(e);
+            tl_last_path = MIPGEMM_PATH_SKINNY | path_flags;
+            return MIPGEMM_OK;
+        }
+    }
+
+    // ---- dense path; operands that TMA cannot address are re-pitched first
+    const bool repack_a = !aligned16(A, lda);
+    const bool repack_b = !aligned16(B, ldb);
+    const long long pitch = round_up(K, 16);
+    Scratch local(dev, stream);
+    Scratch& scratch = outer ? *outer : local;
+    if (!outer && (st = local.reserve(gemm_scratch_bytes(M, N, K, A, lda, B, ldb))) != MIPGEMM_OK) return st;
+    const void* a_use = A;
+    const void* b_use = B;
+    long long lda_use = lda, ldb_use = ldb;
+    if (repack_a) {
+        void* dst = scratch.take(static_cast<size_t>(M) * pitch);
+        cudaError_t e = launch_repack(A, lda, dst, pitch, M, K, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+        a_use = dst;
+        lda_use = pitch;
+        path_flags |= MIPGEMM_PATH_REPACK;
+    }
+    if (repack_b) {
+        void* dst = scratch.take(static_cast<size_t>(N) * pitch);
+        cudaError_t e = launch_repack(B, ldb, dst, pitch, N, K, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+        b_use = dst;
+        ldb_use = pitch;
+        path_flags |= MIPGEMM_PATH_REPACK;
+    }
+
+    const int block_k = 128;
+    const Plan pl = make_plan(M, N, K, block_k, dev->sm_count);
+    DenseParams p;
+    std::memset(&p, 0, sizeof(p));
+    fill_common(p, pl, M, N, C, ldc, block_k, a_unsigned, accumulate, dev);
+    if ((st = encode_tiled_2d(&p.tmap_a, a_use, K, M, lda_use, block_k, kBlockM)) != MIPGEMM_OK) return st;
+    if ((st = encode_tiled_2d(&p.tmap_b, b_use, K, N, ldb_use, block_k, pl.block_n)) != MIPGEMM_OK) return st;
+    if ((st = run_dense(p, pl, M, N, C, ldc, accumulate, dev, stream)) != MIPGEMM_OK) return st;
+    if (pl.split_k > 1) path_flags |= MIPGEMM_PATH_SPLITK;
+    tl_last_path = MIPGEMM_PATH_DENSE | path_flags;
+    return MIPGEMM_OK;
+}
+
+bool conv_geometry(ConvGeom& g) {
+    if (g.Nb < 0 || g.H <= 0 || g.W <= 0 || g.Cin <= 0 || g.Cout < 0 || g.R <= 0 || g.S <= 0) return false;
+    if (g.stride_h <= 0 || g.stride_w <= 0 || g.dil_h <= 0 || g.dil_w <= 0 || g.pad_h < 0 || g.pad_w < 0)
+        return false;
+    const long long eh = g.H + 2LL * g.pad_h - static_cast<long long>(g.dil_h) * (g.R - 1) - 1;
+    const long long ew = g.W + 2LL * g.pad_w - static_cast<long long>(g.dil_w) * (g.S - 1) - 1;
+    if (eh < 0 || ew < 0) return false;
+    g.Ho = eh / g.stride_h + 1;
+    g.Wo = ew / g.stride_w + 1;
+    return true;
+}
+
+bool conv_is_pointwise(const ConvGeom& g) {
+    return g.R == 1 && g.S == 1 && g.stride_h == 1 && g.stride_w == 1 && g.pad_h == 0 && g.pad_w == 0;
+}
+
+// TMA im2col mode: channel count a multiple of the k-block, 16-byte aligned base, and the
+// driver's limits on corners, traversal strides and extents.
+bool conv_tma_eligible(const ConvGeom& g, const void* X, const void* Wt) {
+    if (g.Cin % 64 != 0) return false;
+    if (reinterpret_cast<uintptr_t>(X) % 16 != 0 || reinterpret_cast<uintptr_t>(Wt) % 16 != 0) return false;
+    if (g.stride_h > 8 || g.stride_w > 8) return false;
+    const int lw = -g.pad_w, lh = -g.pad_h;
+    const int uw = g.pad_w - (g.S - 1) * g.dil_w, uh = g.pad_h - (g.R - 1) * g.dil_h;
+    if (lw < -128 || lh < -128 || uw < -128 || uh < -128 || uw > 127 || uh > 127) return false;
+    if ((g.S - 1) * g.dil_w > 65535 || (g.R - 1) * g.dil_h > 65535) return false;
+    if (g.W >= (1LL << 31) || g.H >= (1LL << 31) || g.Nb >= (1LL << 31)) return false;
+    if (g.H * g.W * g.Cin >= (1LL << 40)) return false;
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mipgemm_s8s8s32(int64_t M, int64_t N, int64_t K, const int8_t* A, int64_t lda, const int8_t* B,
+                    int64_t ldb, int32_t* C, int64_t ldc, int accumulate, void* stream) {
+    return gemm_impl(false, M, N, K, A, lda, B, ldb, C, ldc, accumulate, stream, 0);
+}
+
+int mipgemm_u8s8s32(int64_t M, int64_t N, int64_t K, const uint8_t* A, int64_t lda, const int8_t* B,
+                    int64_t ldb, int32_t* C, int64_t ldc, int accumulate, void* stream) {
+    return gemm_impl(true, M, N, K, A, lda, B, ldb, C, ldc, accumulate, stream, 0);
+}
+
+int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int R, int S,
+                         int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                         const uint8_t* X, const int8_t* Wt, int32_t* Y, int accumulate, void* stream_v) {
+    tl_last_path = MIPGEMM_PATH_NONE;
+    ConvGeom g{Nb, H, W, Cin, Cout, 0, 0, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w};
+    if (!conv_geometry(g)) return MIPGEMM_ERR_INVALID_ARG;
+    const long long M = g.Nb * g.Ho * g.Wo;
+    const long long K = static_cast<long long>(R) * S * Cin;
+    if (M > 0x7FFFFF00LL || Cout > 0x7FFFFF00LL) return MIPGEMM_ERR_INVALID_ARG;
+    if (K > 65793) return MIPGEMM_ERR_K_TOO_LARGE;
+    if (M == 0 || Cout == 0) {
+        tl_last_path = MIPGEMM_PATH_TRIVIAL;
+        return MIPGEMM_OK;
+    }
+    if (!X || !Wt || !Y || reinterpret_cast<uintptr_t>(Y) % 4 != 0) return MIPGEMM_ERR_INVALID_ARG;
+
+    if (conv_is_pointwise(g))
+        return gemm_impl(true, M, Cout, Cin, X, Cin, Wt, Cin, Y, Cout, accumulate, stream_v, 0);
+
+    DeviceState* dev = nullptr;
+    int st = get_device(&dev);
+    if (st != MIPGEMM_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+
+    if (conv_tma_eligible(g, X, Wt) && g_tuning.force_path != MIPGEMM_PATH_IM2COL_EXPLICIT) {
+        const int block_k = (Cin % 128 == 0) ? 128 : 64;
+        const Plan pl = make_plan(M, Cout, K, block_k, dev->sm_count);
+        DenseParams p;
+        std::memset(&p, 0, sizeof(p));
+        fill_common(p, pl, M, Cout, Y, Cout, block_k, true, accumulate, dev);
+        p.a_im2col = 1;
+        p.conv_wo = static_cast<int>(g.Wo);
+        p.conv_howo = static_cast<int>(g.Ho * g.Wo);
+        p.conv_s = S;
+        p.c_chunks = static_cast<int>(Cin / block_k);
+        p.stride_w = stride_w; p.stride_h = stride_h;
+        p.pad_w = pad_w; p.pad_h = pad_h;
+        p.dil_w = dil_w; p.dil_h = dil_h;
+        if ((st = encode_im2col(&p.tmap_a, X, g, block_k, kBlockM)) != MIPGEMM_OK) return st;
+        if ((st = encode_tiled_2d(&p.tmap_b, Wt, K, Cout, K, block_k, pl.block_n)) != MIPGEMM_OK) return st;
+        if ((st = run_dense(p, pl, M, Cout, Y, Cout, accumulate, dev, stream)) != MIPGEMM_OK) return st;
+        tl_last_path = MIPGEMM_PATH_DENSE | MIPGEMM_PATH_IM2COL_TMA | (pl.split_k > 1 ? MIPGEMM_PATH_SPLITK : 0);
+        return MIPGEMM_OK;
+    }
+
+    // Explicit lowering: materialise the augmented matrix (zero-padded to a 16-byte pitch),
+    // then run the GEMM on it.  The weight matrix is re-pitched by the GEMM if K % 16 != 0.
+    const long long k_pitch = round_up(K, 16);
+    Scratch scratch(dev, stream);
+    const size_t cols_bytes = align256(static_cast<size_t>(M) * k_pitch);
+    if ((st = scratch.reserve(cols_bytes + gemm_scratch_bytes(M, Cout, K, nullptr, k_pitch, Wt, K))) != MIPGEMM_OK)
+        return st;
+    uint8_t* cols = static_cast<uint8_t*>(scratch.take(static_cast<size_t>(M) * k_pitch));
+    Im2colParams ip{X, cols, g.Nb, g.H, g.W, g.Cin, g.Ho, g.Wo, R, S, stride_h, stride_w,
+                    pad_h, pad_w, dil_h, dil_w, K, k_pitch};
+    cudaError_t e = launch_im2col(ip, stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    // The GEMM takes its own share (weight re-pitching when K % 16 != 0) from the same lease.
+    return gemm_impl(true, M, Cout, K, cols, k_pitch, Wt, K, Y, Cout, accumulate, stream_v,
+                     MIPGEMM_PATH_IM2COL_EXPLICIT, &scratch);
+}
+
+int mipgemm_device_status(void* stream_v) {
+    DeviceState* dev = nullptr;
+    int st = get_device(&dev);
+    if (st != MIPGEMM_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    cudaError_t e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    unsigned int word = 0;
+    e = cudaMemcpy(&word, dev->status_word, sizeof(word), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (word != 0) {
+        e = cudaMemset(dev->status_word, 0, sizeof(word));
+        if (e != cudaSuccess) return cuda_fail(e);
+        return MIPGEMM_ERR_TIMEOUT;
+    }
+    return MIPGEMM_OK;
+}
+
+int mipgemm_set_workspace(void* dev_ptr, size_t bytes) {
+    DeviceState* dev = nullptr;
+    int st = get_device(&dev);
+    if (st != MIPGEMM_OK) return st;
+    if (dev_ptr && reinterpret_cast<uintptr_t>(dev_ptr) % 256 != 0) return MIPGEMM_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    dev->lent = dev_ptr;
+    dev->lent_bytes = dev_ptr ? bytes : 0;
+    return MIPGEMM_OK;
+}
+
+size_t mipgemm_workspace_query_gemm(int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                                    const void* B, int64_t ldb, const void* C, int64_t ldc, int accumulate) {
+    (void)C; (void)ldc; (void)accumulate;
+    return gemm_scratch_bytes(M, N, K, A, lda, B, ldb);
+}
+
+size_t mipgemm_workspace_query_conv(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int R, int S,
+                                    int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w) {
+    ConvGeom g{Nb, H, W, Cin, Cout, 0, 0, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w};
+    if (!conv_geometry(g)) return 0;
+    // Assumes 16-byte aligned tensors (any cudaMalloc'ed or framework-allocated buffer).
+    const long long M = g.Nb * g.Ho * g.Wo;
+    if (conv_is_pointwise(g)) return gemm_scratch_bytes(M, Cout, Cin, nullptr, Cin, nullptr, Cin);
+    if (conv_tma_eligible(g, nullptr, nullptr)) return 0;
+    const long long K = static_cast<long long>(R) * S * Cin;
+    const long long k_pitch = round_up(K, 16);
+    return align256(static_cast<size_t>(M) * k_pitch) + gemm_scratch_bytes(M, Cout, K, nullptr, k_pitch, nullptr, K);
+}
+
+int mipgemm_last_path(void) { return tl_last_path; }
+int mipgemm_last_cuda_error(void) { return tl_last_cuda_error; }
+
+const char* mipgemm_status_string(int status) {
+    switch (status) {
+        case MIPGEMM_OK: return "ok";
+        case MIPGEMM_ERR_INVALID_ARG: return "invalid argument";
+        case MIPGEMM_ERR_K_TOO_LARGE: return "K too large for a guaranteed exact int32 result";
+        case MIPGEMM_ERR_UNSUPPORTED: return "device is not compute capability 10.0 (sm_100a)";
+        case MIPGEMM_ERR_WORKSPACE: return "scratch memory unavailable or lent buffer too small";
+        case MIPGEMM_ERR_CUDA: return "CUDA call failed";
+        case MIPGEMM_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+int mipgemm_version(void) { return 100; }
+
+int mipgemm_probe_i8_peak(int iters, int* grid_out, double* ops_per_launch, int32_t* sink, void* stream_v) {
+    if (iters <= 0 || !sink) return MIPGEMM_ERR_INVALID_ARG;
+    DeviceState* dev = nullptr;
+    int st = get_device(&dev);
+    if (st != MIPGEMM_OK) return st;
+    const int grid = dev->sm_count;
+    cudaError_t e = launch_probe(iters, grid, sink, static_cast<cudaStream_t>(stream_v));
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (grid_out) *grid_out = grid;
+    if (ops_per_launch) *ops_per_launch = 2.0 * 128 * 256 * 128 * static_cast<double>(iters) * grid;
+    return MIPGEMM_OK;
+}
+
+int mipgemm_set_tuning(int block_n, int stages, int split_k, int force_path) {
+    if (block_n != 0 && (block_n < 32 || block_n > 256 || block_n % 32 != 0)) return MIPGEMM_ERR_INVALID_ARG;
+    if (stages < 0 || stages > mip::kMaxStages || split_k < 0) return MIPGEMM_ERR_INVALID_ARG;
+    g_tuning.block_n = block_n;
+    g_tuning.stages = stages;
+    g_tuning.split_k = split_k;
+    g_tuning.force_path = force_path;
+    return MIPGEMM_OK;
+}
+
+}  // extern "C"

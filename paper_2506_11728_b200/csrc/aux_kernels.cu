@@ -1,0 +1,212 @@
+// Auxiliary kernels of libmipgemm: operand re-pitching (the paper's packing step,
+// reborn only to satisfy TMA's 16-byte alignment rule), zero fill of C, explicit
+// im2col for convolutions TMA cannot gather (Section 7.2 lowering), and the
+// tensor-pipe issue-rate probe (the analogue of the Table 1 micro-benchmarks).
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace mip {
+
+// ---------------------------------------------------------------- repack
+// dst[r][0..cols) = src[r][0..cols); dst is 16-byte aligned with a pitch that is a
+// multiple of 16, src has byte alignment only.  Each thread assembles 16 bytes from
+// aligned 32-bit words; only words holding at least one valid byte are read.
+__global__ void mip_repack_kernel(const uint8_t* __restrict__ src, long long src_pitch,
+                                  uint8_t* __restrict__ dst, long long dst_pitch,
+                                  long long rows, long long chunks_per_row, long long cols) {
+    const long long total = rows * chunks_per_row;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long r = i / chunks_per_row;
+        const long long c = (i - r * chunks_per_row) * 16;
+        const int nvalid = static_cast<int>(min(16LL, cols - c));
+        const uint8_t* s = src + r * src_pitch + c;
+        const unsigned off = static_cast<unsigned>(reinterpret_cast<uintptr_t>(s) & 3u);
+        const uint32_t* w = reinterpret_cast<const uint32_t*>(s - off);
+        const int nwords = (static_cast<int>(off) + nvalid + 3) >> 2;
+        uint32_t x[5];
+#pragma unroll
+        for (int j = 0; j < 5; ++j) x[j] = (j < nwords) ? __ldg(w + j) : 0u;
+        uint4 o;
+        o.x = __funnelshift_r(x[0], x[1], off * 8);
+        o.y = __funnelshift_r(x[1], x[2], off * 8);
+        o.z = __funnelshift_r(x[2], x[3], off * 8);
+        o.w = __funnelshift_r(x[3], x[4], off * 8);
+        *reinterpret_cast<uint4*>(dst + r * dst_pitch + c) = o;
+    }
+}
+
+cudaError_t launch_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,
+                          long long rows, long long cols, cudaStream_t stream) {
+    if (rows <= 0 || cols <= 0) return cudaSuccess;
+    const long long chunks = (cols + 15) / 16;
+    const long long total = rows * chunks;
+    const int threads = 256;
+    const long long blocks = min((total + threads - 1) / threads, 148LL * 16);
+    mip_repack_kernel<<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
+        static_cast<const uint8_t*>(src), src_pitch, static_cast<uint8_t*>(dst), dst_pitch, rows,
+        chunks, cols);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- zero fill
+__global__ void mip_fill_zero_kernel(int32_t* C, long long ldc, long long M, long long N) {
+    const long long total = M * N;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long r = i / N;
+        C[r * ldc + (i - r * N)] = 0;
+    }
+}
+
+cudaError_t launch_fill_zero(int32_t* C, long long ldc, long long M, long long N, cudaStream_t stream) {
+    if (M <= 0 || N <= 0) return cudaSuccess;
+    const int threads = 256;
+    const long long blocks = min((M * N + threads - 1) / threads, 148LL * 16);
+    mip_fill_zero_kernel<<<static_cast<unsigned>(blocks), threads, 0, stream>>>(C, ldc, M, N);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- explicit im2col
+// out[m][k], m = ((n*Ho + ho)*Wo + wo), k = (r*S + s)*Cin + c; taps outside the image and
+// the pitch padding k >= k_real are zero.  One thread produces 16 consecutive k.
+template <bool kVec>
+__global__ void mip_im2col_kernel(const Im2colParams p, long long chunks_per_row, long long total) {
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long m = i / chunks_per_row;
+        const long long k0 = (i - m * chunks_per_row) * 16;
+        const long long n = m / (p.Ho * p.Wo);
+        const long long rem = m - n * (p.Ho * p.Wo);
+        const long long ho = rem / p.Wo;
+        const long long wo = rem - ho * p.Wo;
+        const long long hbase = ho * p.stride_h - p.pad_h;
+        const long long wbase = wo * p.stride_w - p.pad_w;
+        uint4 o = make_uint4(0, 0, 0, 0);
+        if (kVec) {
+            // Cin % 16 == 0: the 16 bytes sit inside one tap and are 16-byte aligned in X.
+            if (k0 < p.k_real) {
+                const long long tap = k0 / p.Cin;
+                const long long c = k0 - tap * p.Cin;
+                const long long r = tap / p.S, s = tap - r * p.S;
+                const long long h = hbase + r * p.dil_h, w = wbase + s * p.dil_w;
+                if (h >= 0 && h < p.H && w >= 0 && w < p.W)
+                    o = __ldg(reinterpret_cast<const uint4*>(p.X + ((n * p.H + h) * p.W + w) * p.Cin + c));
+            }
+        } else {
+            uint32_t words[4] = {0, 0, 0, 0};
+            long long tap = k0 / p.Cin;
+            long long c = k0 - tap * p.Cin;
+            long long r = tap / p.S, s = tap - r * p.S;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                if (k0 + j < p.k_real) {
+                    const long long h = hbase + r * p.dil_h, w = wbase + s * p.dil_w;
+                    uint32_t v = 0;
+                    if (h >= 0 && h < p.H && w >= 0 && w < p.W)
+                        v = __ldg(p.X + ((n * p.H + h) * p.W + w) * p.Cin + c);
+                    words[j >> 2] |= v << (8 * (j & 3));
+                    if (++c == p.Cin) {
+                        c = 0;
+                        if (++s == p.S) { s = 0; ++r; }
+                    }
+                }
+            }
+            o = make_uint4(words[0], words[1], words[2], words[3]);
+        }
+        *reinterpret_cast<uint4*>(p.out + m * p.k_pitch + k0) = o;
+    }
+}
+
+cudaError_t launch_im2col(const Im2colParams& p, cudaStream_t stream) {
+    const long long M = p.Nb * p.Ho * p.Wo;
+    if (M <= 0) return cudaSuccess;
+    const long long chunks = p.k_pitch / 16;
+    const long long total = M * chunks;
+    const int threads = 256;
+    const long long blocks = min((total + threads - 1) / threads, 148LL * 32);
+    const bool vec = (p.Cin % 16 == 0) && (reinterpret_cast<uintptr_t>(p.X) % 16 == 0);
+    if (vec)
+        mip_im2col_kernel<true><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(p, chunks, total);
+    else
+        mip_im2col_kernel<false><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(p, chunks, total);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- tensor-pipe probe
+// Every CTA keeps one 128x128-byte A tile and one 256x128-byte B tile (pseudo-random
+// bytes) in shared memory and issues iters*4 MMAs of shape 128x256x32 into two
+// alternating accumulators.  No global traffic inside the loop.
+__global__ void __launch_bounds__(128, 1) mip_probe_kernel(int iters, int32_t* sink) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
+    uint8_t* smem = smem_raw + pad;
+    const uint32_t smem_base = raw_addr + pad;
+    constexpr uint32_t kABytes = 128 * 128, kBBytes = 256 * 128;
+    const uint32_t bar = smem_base + kABytes + kBBytes;
+    uint32_t* slot = reinterpret_cast<uint32_t*>(smem + kABytes + kBBytes + 8);
+
+    uint32_t h = 0x9E3779B9u * (threadIdx.x + 1) + blockIdx.x;
+    for (uint32_t i = threadIdx.x; i < (kABytes + kBBytes) / 4; i += blockDim.x) {
+        h = h * 1664525u + 1013904223u;
+        reinterpret_cast<uint32_t*>(smem)[i] = h ^ (h >> 15);
+    }
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        fence_mbar_init();
+    }
+    fence_proxy_async();
+    if (threadIdx.x < 32) {
+        tmem_alloc<1>(smem_u32(slot), 512);
+        tmem_relinquish<1>();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *slot;
+    bool done = true;
+    if (threadIdx.x == 0) {
+        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+        const uint64_t a_desc = make_kmajor_desc(smem_base, 128);
+        const uint64_t b_desc = make_kmajor_desc(smem_base + kABytes, 128);
+        for (int it = 0; it < iters; ++it) {
+            const uint32_t d = tmem_base + (it & 1) * 256;
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k)
+                mma_i8<1>(d, a_desc + 2ull * k, b_desc + 2ull * k, idesc, (it > 1 || k > 0) ? 1u : 0u);
+        }
+        mma_commit(bar);
+        const uint64_t t0 = globaltimer_ns();
+        while (!mbar_try_wait(bar, 0)) {
+            if (globaltimer_ns() - t0 > 4000000000ull) { done = false; break; }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        tc_fence_after();
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base, v);
+        tmem_ld_wait();
+        if (threadIdx.x == 0) sink[blockIdx.x] = static_cast<int32_t>(v[0]) + (done ? 0 : 1);
+        tc_fence_before();
+        __syncwarp();
+        tmem_dealloc<1>(tmem_base, 512);
+    }
+}
+
+cudaError_t launch_probe(int iters, int grid, int32_t* sink, cudaStream_t stream) {
+    const size_t smem = 128 * 128 + 256 * 128 + 64 + 1024;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(mip_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    mip_probe_kernel<<<grid, 128, smem, stream>>>(iters, sink);
+    return cudaGetLastError();
+}
+
+}  // namespace mip

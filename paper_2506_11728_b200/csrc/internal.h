@@ -1,0 +1,71 @@
+// Host-side declarations shared by the translation units of libmipgemm.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+namespace mip {
+
+constexpr int kBlockM = 128;          // rows of C per CTA (TMEM lanes)
+constexpr int kDenseThreads = 192;    // producer warp, MMA warp, 4 epilogue warps
+constexpr int kMaxStages = 12;
+constexpr int kCtrlBytes = 512;       // barriers + TMEM slot + abort word
+constexpr int kSmemBudget = 227 * 1024;
+
+// Everything the dense kernel needs; passed by value as a __grid_constant__.
+struct alignas(64) DenseParams {
+    CUtensorMap tmap_a;      // tiled {K, M} byte tensor, or im2col-mode NHWC tensor
+    CUtensorMap tmap_b;      // tiled {K, N} byte tensor (weights, K contiguous)
+    int32_t* C;
+    long long ldc;
+    int M, N;
+    int k_blocks;            // ceil(K / block_k)
+    int block_n;             // multiple of 32, <= 256
+    int block_k;             // bytes of K per pipeline stage: 128 (SWIZZLE_128B) or 64 (SWIZZLE_64B)
+    int stages;
+    int tiles_m, tiles_n;
+    int split_k, kb_per_split;
+    int group_n;             // n-tiles per rasterisation group
+    int accumulate;          // epilogue adds the incoming C
+    int use_red;             // epilogue reduces with red.global.add (split-K)
+    int store_vec;           // 8, 4 or 1 int32 per store instruction
+    uint32_t idesc;          // tcgen05 instruction descriptor
+    uint32_t tmem_cols;      // power of two >= 2*block_n
+    // implicit im2col (operand A gathered by TMA im2col loads)
+    int a_im2col;
+    int conv_wo, conv_howo, conv_s, c_chunks;
+    int stride_w, stride_h, pad_w, pad_h, dil_w, dil_h;
+    unsigned int* status;    // device word, bit 0 set when a bounded wait expired
+    unsigned long long wait_budget_ns;
+};
+
+cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream);
+cudaError_t launch_dense_pair(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream);
+cudaError_t dense_init();  // opt in to large dynamic shared memory (once per device)
+
+// Skinny-M streaming kernel (M <= 16).
+struct SkinnyParams {
+    const void* A; long long lda;
+    const int8_t* B; long long ldb;
+    int32_t* C; long long ldc;
+    int M, N, K;
+    int a_unsigned, accumulate;
+};
+cudaError_t launch_skinny(const SkinnyParams& p, cudaStream_t stream);
+bool skinny_supported(const SkinnyParams& p);
+
+// Auxiliary kernels.
+cudaError_t launch_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,
+                          long long rows, long long cols, cudaStream_t stream);
+cudaError_t launch_fill_zero(int32_t* C, long long ldc, long long M, long long N, cudaStream_t stream);
+struct Im2colParams {
+    const uint8_t* X; uint8_t* out;
+    long long Nb, H, W, Cin, Ho, Wo;
+    int R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
+    long long k_real, k_pitch;   // R*S*Cin and its padded pitch (pad bytes are zero-filled)
+};
+cudaError_t launch_im2col(const Im2colParams& p, cudaStream_t stream);
+cudaError_t launch_probe(int iters, int grid, int32_t* sink, cudaStream_t stream);
+
+}  // namespace mip

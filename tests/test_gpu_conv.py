@@ -1,0 +1,111 @@
+"""GPU parity for the convolution entry point against the direct-convolution oracle."""
+import numpy as np
+import pytest
+
+from oracle import mip_oracle as orc
+from paper_2506_11728_b200 import inputs
+from gpu_util import run_conv, first_mismatch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mg():
+    from paper_2506_11728_b200 import binding
+    binding.mipgemm_set_tuning()
+    return binding
+
+
+def conv_inputs(Nb, H, W, Cin, Cout, R, S, seed):
+    X = inputs.uniform_u8(Nb * H * W * Cin, seed + 1).reshape(Nb, H, W, Cin)
+    Wt = inputs.normal_s8(Cout * R * S * Cin, seed + 2, 32.0, -127, 127).reshape(Cout, R, S, Cin)
+    return X, Wt
+
+
+def check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil=(1, 1), seed=0, accumulate=False,
+               expect_flag=None):
+    X, Wt = conv_inputs(Nb, H, W, Cin, Cout, R, S, seed)
+    Y0 = None
+    if accumulate:
+        Ho, Wo = orc.conv_out_hw(H, W, R, S, stride, pad, dil)
+        Y0 = inputs.uniform_s32(Nb * Ho * Wo * Cout, seed + 3).reshape(Nb, Ho, Wo, Cout)
+    want = orc.conv(X, Wt, stride=stride, pad=pad, dil=dil, Y=None if Y0 is None else Y0.copy(),
+                    accumulate=accumulate)
+    got, path = run_conv(mg, X, Wt, stride, pad, dil, Y=None if Y0 is None else Y0.copy(),
+                         accumulate=accumulate)
+    assert np.array_equal(got, want), "conv %s path=%#x: %s" % (
+        (Nb, H, W, Cin, Cout, R, S, stride, pad, dil), path, first_mismatch(got, want))
+    if expect_flag is not None:
+        assert path & expect_flag, hex(path)
+    return path
+
+
+def test_pointwise_is_plain_gemm(mg):
+    p = check_conv(mg, 2, 14, 14, 256, 96, 1, 1, (1, 1), (0, 0), seed=1)
+    assert not p & (mg.PATH_IM2COL_TMA | mg.PATH_IM2COL_EXPLICIT)
+    check_conv(mg, 3, 7, 9, 24, 40, 1, 1, (1, 1), (0, 0), seed=2)            # Cin % 16 != 0 -> repack
+
+
+TMA_CASES = [
+    # Nb, H, W, Cin, Cout, R, S, stride, pad, dil
+    (2, 14, 14, 128, 128, 3, 3, (1, 1), (1, 1), (1, 1)),
+    (2, 28, 28, 128, 64, 3, 3, (2, 2), (1, 1), (1, 1)),
+    (3, 13, 11, 64, 64, 3, 3, (1, 1), (1, 1), (1, 1)),       # 64-byte k-block, odd extents
+    (2, 16, 16, 256, 160, 1, 1, (2, 2), (0, 0), (1, 1)),     # strided 1x1 (projection shortcut)
+    (1, 20, 18, 128, 96, 3, 3, (1, 1), (2, 2), (2, 2)),      # dilation
+    (2, 15, 17, 128, 72, 5, 3, (2, 1), (2, 1), (1, 1)),      # rectangular filter, mixed stride
+    (5, 7, 7, 512, 512, 3, 3, (1, 1), (1, 1), (1, 1)),       # tiles straddle images; K = 4608
+    (1, 9, 9, 128, 64, 3, 3, (1, 1), (0, 0), (1, 1)),        # no padding
+]
+
+
+@pytest.mark.parametrize("case", TMA_CASES)
+def test_implicit_im2col_tma(mg, case):
+    Nb, H, W, Cin, Cout, R, S, stride, pad, dil = case
+    check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=10, expect_flag=mg.PATH_IM2COL_TMA)
+    check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=11, accumulate=True,
+               expect_flag=mg.PATH_IM2COL_TMA)
+
+
+EXPLICIT_CASES = [
+    (2, 32, 32, 3, 64, 7, 7, (2, 2), (3, 3), (1, 1)),        # stem-like, Cin = 3, K = 147
+    (2, 12, 12, 16, 32, 3, 3, (1, 1), (1, 1), (1, 1)),       # Cin % 16 == 0 but not % 64
+    (1, 10, 11, 5, 7, 3, 2, (2, 1), (1, 0), (1, 2)),
+]
+
+
+@pytest.mark.parametrize("case", EXPLICIT_CASES)
+def test_explicit_im2col(mg, case):
+    Nb, H, W, Cin, Cout, R, S, stride, pad, dil = case
+    check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=20, expect_flag=mg.PATH_IM2COL_EXPLICIT)
+    check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=21, accumulate=True,
+               expect_flag=mg.PATH_IM2COL_EXPLICIT)
+
+
+def test_forced_explicit_matches_tma(mg):
+    case = TMA_CASES[1]
+    Nb, H, W, Cin, Cout, R, S, stride, pad, dil = case
+    mg.mipgemm_set_tuning(force_path=mg.PATH_IM2COL_EXPLICIT)
+    try:
+        check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=30, expect_flag=mg.PATH_IM2COL_EXPLICIT)
+    finally:
+        mg.mipgemm_set_tuning()
+
+
+@pytest.mark.parametrize("layer", range(len(inputs.RESNET50_CONVS)))
+def test_resnet50_layers_batch2_full(mg, layer):
+    _cnt, H, W, Cin, Cout, R, S, st, pd = inputs.RESNET50_CONVS[layer]
+    check_conv(mg, 2, H, W, Cin, Cout, R, S, (st, st), (pd, pd), seed=inputs.seed_for(3, layer))
+
+
+@pytest.mark.parametrize("layer", [0, 2, 6, 8, 16, 18, 22])
+def test_resnet50_layers_batch32_sampled_images(mg, layer):
+    """Full batch on the GPU; the oracle recomputes two whole images (the output of image n
+    depends on image n only) -- first and last, so tile runs that cross image borders count."""
+    _cnt, H, W, Cin, Cout, R, S, st, pd = inputs.RESNET50_CONVS[layer]
+    Nb = 32
+    X, Wt = conv_inputs(Nb, H, W, Cin, Cout, R, S, inputs.seed_for(3, layer))
+    got, _ = run_conv(mg, X, Wt, (st, st), (pd, pd), (1, 1))
+    for n in (0, 17, Nb - 1):
+        want = orc.conv(X[n:n + 1], Wt, stride=(st, st), pad=(pd, pd))
+        assert np.array_equal(got[n:n + 1], want), "image %d: %s" % (n, first_mismatch(got[n:n + 1], want))

@@ -1,0 +1,223 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, bit for bit."""
+import numpy as np
+import pytest
+
+from oracle import mip_oracle as orc
+from paper_2506_11728_b200 import inputs
+from gpu_util import run_gemm, first_mismatch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mg():
+    from paper_2506_11728_b200 import binding
+    binding.mipgemm_set_tuning()
+    return binding
+
+
+def make_ab(mode, M, N, K, lda, ldb, seed, dist="uniform"):
+    if dist == "uniform":
+        A = inputs.uniform_s8(M * lda, seed + 1) if mode == "s8" else inputs.uniform_u8(M * lda, seed + 1)
+        B = inputs.uniform_s8(N * ldb, seed + 2)
+    else:
+        A = inputs.normal_s8(M * lda, seed + 1, 40.0)
+        B = inputs.normal_s8(N * ldb, seed + 2, 20.0)
+    return A, B
+
+
+def check_case(mg, mode, M, N, K, *, lda=None, ldb=None, ldc=None, accumulate=False, seed=0,
+               misalign_a=0, misalign_b=0, expect_path=None, dist="uniform"):
+    lda = K if lda is None else lda
+    ldb = K if ldb is None else ldb
+    ldc = N if ldc is None else ldc
+    A, B = make_ab(mode, M, N, K, lda, ldb, seed, dist)
+    if accumulate:
+        C0 = inputs.uniform_s32(M * ldc, seed + 3)
+    else:
+        C0 = np.full(M * ldc, 0x7F7F7F7F, dtype=np.int32)
+    want = orc.gemm(A, B, M, N, K, lda=lda, ldb=ldb, C=C0.copy(), ldc=ldc, accumulate=accumulate)
+    got, path = run_gemm(mg, mode, M, N, K, A, B, lda=lda, ldb=ldb, C=C0.copy(), ldc=ldc,
+                         accumulate=accumulate, misalign_a=misalign_a, misalign_b=misalign_b,
+                         expect_path=expect_path)
+    # padding columns included: they must still hold what C0 held
+    assert np.array_equal(got[:M * ldc], want), "%s M=%d N=%d K=%d acc=%d path=%#x: %s" % (
+        mode, M, N, K, accumulate, path, first_mismatch(got[:M * ldc].reshape(M, ldc), want.reshape(M, ldc)))
+    return path
+
+
+def test_config1_512_cubed(mg):
+    check_case(mg, "s8", 512, 512, 512, seed=inputs.seed_for(1, 0), expect_path=mg.PATH_DENSE)
+    # BASELINE wording: zero-initialised C, accumulate=0 -- and accumulate onto it gives the same
+    A, B = make_ab("s8", 512, 512, 512, 512, 512, inputs.seed_for(1, 0))
+    want = orc.gemm(A, B, 512, 512, 512)
+    got, _ = run_gemm(mg, "s8", 512, 512, 512, A, B, C=np.zeros(512 * 512, np.int32), accumulate=True)
+    assert np.array_equal(got, want)
+
+
+RAGGED = [
+    (17, 16, 16), (128, 256, 128), (129, 257, 144), (127, 255, 112), (1, 1, 16), (33, 7, 48),
+    (200, 40, 1040), (256, 512, 384), (255, 513, 400), (300, 100, 2048), (77, 300, 16),
+    (640, 96, 272), (130, 130, 130 // 16 * 16 + 16),
+]
+
+
+@pytest.mark.parametrize("mode", ["s8", "u8"])
+@pytest.mark.parametrize("accumulate", [False, True])
+def test_ragged_shapes_dense(mg, mode, accumulate):
+    mg.mipgemm_set_tuning(force_path=mg.PATH_DENSE)
+    try:
+        for i, (M, N, K) in enumerate(RAGGED):
+            check_case(mg, mode, M, N, K, accumulate=accumulate, seed=100 + i, expect_path=mg.PATH_DENSE)
+    finally:
+        mg.mipgemm_set_tuning()
+
+
+@pytest.mark.parametrize("block_n", [64, 128, 256, 96])
+def test_tile_widths_and_pitches(mg, block_n):
+    mg.mipgemm_set_tuning(block_n=block_n)
+    try:
+        check_case(mg, "s8", 300, 700, 400, lda=416, ldb=432, ldc=708, seed=7)       # ldc % 4 == 0
+        check_case(mg, "u8", 300, 700, 400, lda=400, ldb=400, ldc=705, seed=8, accumulate=True)  # scalar stores
+        check_case(mg, "s8", 260, 520, 272, ldc=520, seed=9)
+    finally:
+        mg.mipgemm_set_tuning()
+
+
+@pytest.mark.parametrize("stages", [2, 3])
+def test_shallow_pipelines_wrap_phases(mg, stages):
+    mg.mipgemm_set_tuning(block_n=128, stages=stages)
+    try:
+        check_case(mg, "s8", 700, 600, 1424, seed=11)
+    finally:
+        mg.mipgemm_set_tuning()
+
+
+def test_many_tiles_per_cta_persistent_loop(mg):
+    # 32 x 16 = 512 tiles of 128x128 on 148 CTAs: 3-4 tiles per CTA, both accumulators reused
+    mg.mipgemm_set_tuning(block_n=128)
+    try:
+        check_case(mg, "s8", 4096, 2048, 256, seed=13)
+    finally:
+        mg.mipgemm_set_tuning()
+
+
+def test_misaligned_operands_take_the_repack_path(mg):
+    # config 2b: every pitch odd, accumulate onto a seeded C
+    path = check_case(mg, "s8", 1000, 3001, 777, lda=777, ldb=777, ldc=3001, accumulate=True,
+                      seed=inputs.seed_for(2, 0))
+    assert path & mg.PATH_REPACK
+    path = check_case(mg, "u8", 130, 70, 100, lda=101, ldb=103, ldc=71, seed=21)
+    assert path & mg.PATH_REPACK
+    # aligned pitches but misaligned base pointers
+    path = check_case(mg, "s8", 140, 90, 160, misalign_a=3, misalign_b=5, seed=22)
+    assert path & mg.PATH_REPACK
+    path = check_case(mg, "s8", 5, 9, 13, seed=23)                                  # tiny, K % 16 != 0
+    assert path & mg.PATH_REPACK
+
+
+def test_split_k_reduction(mg):
+    path = check_case(mg, "s8", 128, 256, 8192, seed=31)
+    assert path & mg.PATH_SPLITK
+    path = check_case(mg, "u8", 200, 100, 4096 + 48, accumulate=True, seed=32)
+    assert path & mg.PATH_SPLITK
+    mg.mipgemm_set_tuning(split_k=5)
+    try:
+        check_case(mg, "s8", 300, 300, 1296, ldc=301, seed=33)
+    finally:
+        mg.mipgemm_set_tuning()
+
+
+def test_k_zero_and_empty(mg):
+    M, N = 37, 21
+    A = np.zeros(16, np.int8)
+    B = np.zeros(16, np.int8)
+    C0 = inputs.uniform_s32(M * (N + 3), 5)
+    got, path = run_gemm(mg, "s8", M, N, 0, A, B, lda=0, ldb=0, C=C0.copy(), ldc=N + 3, accumulate=False)
+    want = C0.reshape(M, N + 3).copy()
+    want[:, :N] = 0
+    assert np.array_equal(got.reshape(M, N + 3), want) and path & mg.PATH_MASK == mg.PATH_TRIVIAL
+    got, _ = run_gemm(mg, "s8", M, N, 0, A, B, lda=0, ldb=0, C=C0.copy(), ldc=N + 3, accumulate=True)
+    assert np.array_equal(got, C0)
+
+
+@pytest.mark.parametrize("mode,a_val,b_val,per_k", [
+    ("s8", -128, -128, 16384), ("s8", -128, 127, -16256), ("u8", 255, -128, -32640), ("u8", 255, 127, 32385)])
+def test_extreme_values_closed_form(mg, mode, a_val, b_val, per_k):
+    M, N, K = 256, 384, 2048
+    A = np.full(M * K, a_val, dtype=np.int8 if mode == "s8" else np.uint8)
+    B = np.full(N * K, b_val, dtype=np.int8)
+    got, _ = run_gemm(mg, mode, M, N, K, A, B)
+    assert (got == per_k * K).all()
+
+
+def test_largest_exact_k(mg):
+    # the K limits of the exactness contract, at the worst-case operand values
+    for mode, K, a_val, expect in (("s8", 131071 // 16 * 16, -128, None), ("u8", 65793 // 16 * 16, 255, None)):
+        M, N = 128, 64
+        A = np.full(M * K, a_val, dtype=np.int8 if mode == "s8" else np.uint8)
+        B = np.full(N * K, -128, dtype=np.int8)
+        got, _ = run_gemm(mg, mode, M, N, K, A, B)
+        assert (got.astype(np.int64) == int(a_val) * -128 * K).all()
+
+
+def test_square_sweep_small_members_full_oracle(mg):
+    for n in (1024, 2048):
+        check_case(mg, "s8", n, n, n, seed=inputs.seed_for(2, n))
+    n = 1024
+    A = np.full(n * n, -128, np.int8)
+    got, _ = run_gemm(mg, "s8", n, n, n, A, A)
+    assert (got == 16384 * n).all()
+
+
+BERT_T1024 = [(1024, N, K) for (_name, N, K) in inputs.BERT_GEMMS]
+
+
+@pytest.mark.parametrize("shape", BERT_T1024)
+def test_bert_shapes_t1024(mg, shape):
+    M, N, K = shape
+    check_case(mg, "s8", M, N, K, seed=inputs.seed_for(4, N + K), dist="normal")
+
+
+@pytest.mark.parametrize("M", inputs.SKINNY_M)
+@pytest.mark.parametrize("mode", ["s8", "u8"])
+def test_skinny_small(mg, M, mode):
+    for (N, K) in [(16, 16), (100, 272), (1000, 1040), (4096 + 7, 4096)]:
+        for acc in (False, True):
+            check_case(mg, mode, M, N, K, accumulate=acc, seed=200 + M, ldc=N + 1, expect_path=mg.PATH_SKINNY)
+    # other M <= 16
+    for Mx in (2, 3, 7, 9, 15):
+        check_case(mg, mode, Mx, 333, 528, seed=300 + Mx, expect_path=mg.PATH_SKINNY)
+
+
+@pytest.mark.parametrize("NK", inputs.SKINNY_WEIGHTS)
+def test_skinny_full_size_weights(mg, NK):
+    N, K = NK
+    for M in (1, 16):
+        check_case(mg, "s8", M, N, K, seed=inputs.seed_for(5, M), expect_path=mg.PATH_SKINNY)
+
+
+def test_skinny_misaligned_falls_back_to_dense(mg):
+    path = check_case(mg, "s8", 4, 300, 100, seed=41)
+    assert path & mg.PATH_MASK == mg.PATH_DENSE and path & mg.PATH_REPACK
+
+
+def test_lent_workspace(mg):
+    import torch
+    need = mg.mipgemm_workspace_query_gemm(130, 70, 100, 0, 101, 0, 103, 0, 71)
+    assert need > 0
+    buf = torch.empty(need, dtype=torch.uint8, device="cuda")
+    assert mg.mipgemm_set_workspace(buf, need) == mg.OK
+    try:
+        check_case(mg, "u8", 130, 70, 100, lda=101, ldb=103, ldc=71, seed=21)
+        small = torch.empty(256, dtype=torch.uint8, device="cuda")
+        mg.mipgemm_set_workspace(small, 256)
+        A = np.zeros(130 * 101, np.uint8)
+        B = np.zeros(70 * 103, np.int8)
+        from gpu_util import to_dev
+        dA, _a = to_dev(A)
+        dB, _b = to_dev(B)
+        dC = torch.zeros(130 * 71, dtype=torch.int32, device="cuda")
+        assert mg.mipgemm_u8s8s32(130, 70, 100, dA, 101, dB, 103, dC, 71, 0, check=False) == mg.ERR_WORKSPACE
+    finally:
+        mg.mipgemm_set_workspace(None, 0)
