@@ -1,0 +1,524 @@
+#!/usr/bin/env python
+"""Benchmark of libmipgemm on B200: one JSON line per run.
+
+A *step* is one pass of the hot path over one batch of synthetic input: every GEMM (or
+convolution) of the chosen workload, launched back to back on one stream through the C
+ABI.  The default workload is the square s8*s8->s32 sweep M=N=K in {1024 .. 16384}.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload square|bert|resnet|skinny]
+    python bench.py --impl reference ...      # the CPU oracle, timed on the host cores
+
+Under torchrun (N > 1) every rank runs the same per-GPU workload on its own device
+(independent problems, no data-path collective: weak scaling); the time is the maximum
+over ranks and the value is the aggregate over all ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2506_11728_b200 import inputs  # noqa: E402  (bytes only, no arithmetic)
+
+NOMINAL_INT8_TOPS = 4500.0
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM traffic (bytes read + written) of the dominant kernel per launch, from the ncu
+# captures summarised under profiles/ (None until a capture exists for that workload).
+NCU_TRAFFIC_BYTES = {"square": None, "bert": None, "resnet": None, "skinny": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+# --------------------------------------------------------------------------- workloads
+class Problem:
+    """One library call: shapes, algorithmic ops/bytes and the device buffers it runs on."""
+
+    def __init__(self, name, kind, ops, nbytes):
+        self.name, self.kind, self.ops, self.bytes = name, kind, float(ops), float(nbytes)
+        self.calls = []          # list of zero-argument callables (one per rotation slot)
+        self.host = None         # host-side operands for the end-to-end leg (gemm only)
+
+    def launch(self, i):
+        self.calls[i % len(self.calls)]()
+
+
+def _dev_bytes(torch, arr):
+    t = torch.from_numpy(arr.view(np.uint8))
+    return t.cuda(non_blocking=False)
+
+
+def build_square(torch, mg, sizes, keep_host):
+    probs = []
+    for n in sizes:
+        A = inputs.uniform_s8(n * n, inputs.seed_for(2, n) + 1)
+        B = inputs.uniform_s8(n * n, inputs.seed_for(2, n) + 2)
+        dA, dB = _dev_bytes(torch, A), _dev_bytes(torch, B)
+        dC = torch.empty(n * n, dtype=torch.int32, device="cuda")
+        p = Problem("square_%d" % n, "gemm", 2.0 * n * n * n, 2.0 * n * n + 4.0 * n * n)
+        p.dims = (n, n, n)
+        p.bufs = (dA, dB, dC)
+        p.calls = [lambda n=n, dA=dA, dB=dB, dC=dC: mg.mipgemm_s8s8s32(n, n, n, dA, n, dB, n, dC, n, 0)]
+        if keep_host:
+            p.host = (A, B)
+        probs.append(p)
+    return probs
+
+
+def build_bert(torch, mg, tokens):
+    probs = []
+    for T in tokens:
+        for (name, N, K) in inputs.BERT_GEMMS:
+            A = inputs.normal_s8(T * K, inputs.seed_for(4, N + K) + 1, 40.0)
+            B = inputs.normal_s8(N * K, inputs.seed_for(4, N + K) + 2, 20.0)
+            dA, dB = _dev_bytes(torch, A), _dev_bytes(torch, B)
+            dC = torch.empty(T * N, dtype=torch.int32, device="cuda")
+            p = Problem("%s_T%d" % (name, T), "gemm", 2.0 * T * N * K, T * K + N * K + 4.0 * T * N)
+            p.dims = (T, N, K)
+            p.bufs = (dA, dB, dC)
+            p.calls = [lambda T=T, N=N, K=K, dA=dA, dB=dB, dC=dC:
+                       mg.mipgemm_s8s8s32(T, N, K, dA, K, dB, K, dC, N, 0)]
+            probs.append(p)
+    return probs
+
+
+def build_resnet(torch, mg, batch):
+    probs = []
+    for li, (cnt, H, W, Cin, Cout, R, S, st, pd) in enumerate(inputs.RESNET50_CONVS):
+        Ho = (H + 2 * pd - (R - 1) - 1) // st + 1
+        Wo = (W + 2 * pd - (S - 1) - 1) // st + 1
+        X = inputs.uniform_u8(batch * H * W * Cin, inputs.seed_for(3, li) + 1)
+        Wt = inputs.normal_s8(Cout * R * S * Cin, inputs.seed_for(3, li) + 2, 32.0, -127, 127)
+        dX, dW = _dev_bytes(torch, X), _dev_bytes(torch, Wt)
+        dY = torch.empty(batch * Ho * Wo * Cout, dtype=torch.int32, device="cuda")
+        M, K = batch * Ho * Wo, R * S * Cin
+        p = Problem("conv%02d_%dx%dx%d_%d_%dx%d_s%d" % (li + 1, H, W, Cin, Cout, R, S, st), "conv",
+                    2.0 * M * Cout * K, batch * H * W * Cin + Cout * K + 4.0 * M * Cout)
+        p.dims = (M, Cout, K)
+        p.count = cnt
+        p.bufs = (dX, dW, dY)
+        p.calls = [lambda a=(batch, H, W, Cin, Cout, R, S, st, st, pd, pd, 1, 1), dX=dX, dW=dW, dY=dY:
+                   mg.mipgemm_conv_u8s8s32(*a, dX, dW, dY, 0)]
+        probs.append(p)
+    return probs
+
+
+def build_skinny(torch, mg, rotate_bytes=512 << 20):
+    probs = []
+    for (N, K) in inputs.SKINNY_WEIGHTS:
+        slots = max(2, -(-rotate_bytes // (N * K)))
+        Bs = []
+        for r in range(slots):
+            Bs.append(_dev_bytes(torch, inputs.uniform_s8(N * K, inputs.seed_for(5, N + K) + 10 * r + 2)))
+        for M in inputs.SKINNY_M:
+            A = inputs.uniform_s8(M * K, inputs.seed_for(5, M) + 1)
+            dA = _dev_bytes(torch, A)
+            dC = torch.empty(M * N, dtype=torch.int32, device="cuda")
+            p = Problem("skinny_M%d_%dx%d" % (M, N, K), "gemm", 2.0 * M * N * K, N * K + M * K + 4.0 * M * N)
+            p.dims = (M, N, K)
+            p.bufs = (dA, Bs, dC)
+            p.calls = [lambda M=M, N=N, K=K, dA=dA, dB=dB, dC=dC:
+                       mg.mipgemm_s8s8s32(M, N, K, dA, K, dB, K, dC, N, 0) for dB in Bs]
+            probs.append(p)
+    return probs
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons through NVML while the timed region runs
+    (read-only queries)."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting"}
+
+    def __init__(self, torch, device_index):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.power = [], set(), []
+        self.stop_flag = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            handle = None
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                handle = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                handle = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.h = handle
+            self.max_sm = int(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as exc:  # NVML missing: report that instead of inventing numbers
+            self.err = repr(exc)
+
+    def _once(self):
+        nv = self.nv
+        self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+        try:
+            getter = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+                nv.nvmlDeviceGetCurrentClocksThrottleReasons
+            mask = int(getter(self.h))
+            for bit, name in self.REASONS.items():
+                if mask & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+        try:
+            self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+        except Exception:
+            pass
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self.stop_flag.is_set():
+            try:
+                self._once()
+            except Exception:
+                break
+            time.sleep(0.004)
+
+    def summary(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML unavailable"}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_sm,
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w_max": max(self.power) if self.power else None}
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample_rows(problems, frac):
+    rows = []
+    for p in problems:
+        M = p.dims[0]
+        rows.append(max(1, min(M, int(round(M * frac)))))
+    return rows
+
+
+def time_oracle_sample(problems, frac, compare_with=None):
+    """Runs the oracle on the first rows of every GEMM of the workload; returns (seconds, ops).
+    If ``compare_with`` maps a problem name to the GPU result, the sampled rows are also
+    compared bit for bit."""
+    from oracle import mip_oracle as orc
+    total_s, total_ops, parity = 0.0, 0.0, None
+    for p, r in zip(problems, oracle_sample_rows(problems, frac)):
+        M, N, K = p.dims
+        A, B = p.host
+        t0 = time.perf_counter()
+        want = orc.gemm(A[:r * K], B, r, N, K)
+        total_s += time.perf_counter() - t0
+        total_ops += 2.0 * r * N * K
+        if compare_with is not None and p.name in compare_with:
+            got = compare_with[p.name][:r * N]
+            same = bool(np.array_equal(got, want))
+            parity = same if parity is None else (parity and same)
+    return total_s, total_ops, parity
+
+
+def calibrate_fraction(problems, target_s):
+    """Sample fraction (of every problem's rows) so the oracle runs for about target_s."""
+    from oracle import mip_oracle as orc
+    p = problems[min(2, len(problems) - 1)]
+    M, N, K = p.dims
+    A, B = p.host
+    r = min(M, 8)
+    orc.gemm(A[:r * K], B, r, N, K)                    # builds / warms the oracle
+    t0 = time.perf_counter()
+    orc.gemm(A[:r * K], B, r, N, K)
+    rate = 2.0 * r * N * K / max(time.perf_counter() - t0, 1e-6)
+    total = sum(q.ops for q in problems)
+    return max(1e-6, min(1.0, target_s * rate / total))
+
+
+def host_only_square(sizes):
+    probs = []
+    for n in sizes:
+        p = Problem("square_%d" % n, "gemm", 2.0 * n * n * n, 6.0 * n * n)
+        p.dims = (n, n, n)
+        p.host = (inputs.uniform_s8(n * n, inputs.seed_for(2, n) + 1),
+                  inputs.uniform_s8(n * n, inputs.seed_for(2, n) + 2))
+        probs.append(p)
+    return probs
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on the host cores: each step a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import mip_oracle as orc
+    sizes = [s for s in inputs.SQUARE_SIZES if s <= args.max_size]
+    probs = host_only_square(sizes)
+    frac = calibrate_fraction(probs, 60.0 / max(1, args.steps + args.warmup))
+    for _ in range(args.warmup):
+        time_oracle_sample(probs, frac)
+    secs, ops = 0.0, 0.0
+    for _ in range(args.steps):
+        s, o, _p = time_oracle_sample(probs, frac)
+        secs += s
+        ops += o
+    value = ops / secs / 1e12
+    rows = oracle_sample_rows(probs, frac)
+    sample = "first rows of every sweep member: " + ", ".join(
+        "%d of %d" % (r, p.dims[0]) for r, p in zip(rows, probs))
+    line = {
+        "impl": "reference", "metric": "int8_gemm_tops", "value": value, "unit": "TOPS",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": "square s8*s8->s32 sweep M=N=K in %s (sampled rows per step)" % sizes},
+        "cpu_baseline": {"value": value, "unit": "TOPS", "cores": orc.threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- main arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="square", choices=["square", "bert", "resnet", "skinny"])
+    ap.add_argument("--max-size", type=int, default=16384, help="largest member of the square sweep")
+    ap.add_argument("--batch", type=int, default=32, help="resnet batch")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--detail", action="store_true", help="print per-problem timings to stderr")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    from paper_2506_11728_b200 import build as _build
+    _build.build_library()
+    from paper_2506_11728_b200 import binding as mg
+
+    want_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline and args.workload == "square")
+    if args.workload == "square":
+        sizes = [s for s in inputs.SQUARE_SIZES if s <= args.max_size]
+        probs = build_square(torch, mg, sizes, keep_host=True)
+        workload = "square s8*s8->s32 sweep M=N=K in %s, uniform int8, accumulate=0" % sizes
+        unit, metric = "TOPS", "int8_gemm_tops"
+    elif args.workload == "bert":
+        probs = build_bert(torch, mg, inputs.BERT_TOKENS)
+        workload = "BERT base/large encoder GEMMs s8*s8->s32, tokens %s" % inputs.BERT_TOKENS
+        unit, metric = "TOPS", "int8_gemm_tops"
+    elif args.workload == "resnet":
+        probs = build_resnet(torch, mg, args.batch)
+        workload = "ResNet-50 v1.5 convolutions u8*s8->s32 NHWC, batch %d, 53 layers" % args.batch
+        unit, metric = "TOPS", "int8_conv_tops"
+    else:
+        probs = build_skinny(torch, mg)
+        workload = "skinny decode GEMMs s8*s8->s32, M in %s, weights %s, rotated over >=512 MB" % (
+            inputs.SKINNY_M, inputs.SKINNY_WEIGHTS)
+        unit, metric = "GB/s", "skinny_gemm_gbs"
+
+    # launch order of one step: every problem once (resnet: layer multiplicity; skinny: all slots)
+    order = []
+    for p in probs:
+        reps = getattr(p, "count", 1) if args.workload == "resnet" else len(p.calls)
+        order.extend([(p, i) for i in range(reps)])
+
+    def one_step(events=None):
+        for j, (p, i) in enumerate(order):
+            if events is not None:
+                events[j][0].record()
+            p.launch(i)
+            if events is not None:
+                events[j][1].record()
+
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        one_step()
+    torch.cuda.synchronize()
+    assert mg.mipgemm_device_status() == mg.OK
+
+    # ---- timed region: exactly K steps between two synchronisation points
+    per_launch = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in order] for _ in range(args.steps)]
+    sampler = ClockSampler(torch, local_rank)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = mg.mipgemm_launch_count()
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for s in range(args.steps):
+        one_step(per_launch[s])
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler.stop_flag.set()
+    sampler.join(timeout=2.0)
+    launches = mg.mipgemm_launch_count() - launches0
+    assert mg.mipgemm_device_status() == mg.OK
+    elapsed_ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+
+    step_ops = sum(p.ops for (p, _i) in order)
+    step_bytes = sum(p.bytes for (p, _i) in order)
+    ms_per_step = elapsed_ms / args.steps
+    if unit == "TOPS":
+        value = world * step_ops / (ms_per_step * 1e-3) / 1e12
+    else:
+        value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- per-problem kernel time from the events recorded inside the timed region
+    agg = {}
+    for s in range(args.steps):
+        for j, (p, _i) in enumerate(order):
+            a, b = per_launch[s][j]
+            d = agg.setdefault(p.name, [0.0, 0, p])
+            d[0] += a.elapsed_time(b)
+            d[1] += 1
+    detail = []
+    for name, (ms, n, p) in agg.items():
+        avg = ms / n
+        detail.append({"name": name, "us": avg * 1e3, "tops": p.ops / (avg * 1e-3) / 1e12,
+                       "gbs": p.bytes / (avg * 1e-3) / 1e9})
+    if args.detail and rank == 0:
+        for d in detail:
+            sys.stderr.write("%-40s %10.1f us %9.1f TOPS %9.1f GB/s\n" % (d["name"], d["us"], d["tops"], d["gbs"]))
+
+    # ---- roofline of the dominant kernel over the timed region
+    peaks = load_peaks()
+    kernel_ms = sum(v[0] for v in agg.values())
+    n_launch = sum(v[1] for v in agg.values())
+    if unit == "TOPS" and args.workload in ("square", "bert"):
+        int8_burst = peaks["bf16_tflops"] * (NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS)
+        int8_sust = peaks["bf16_tflops_sustained"] * (NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS)
+        achieved = args.steps * step_ops / (kernel_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "mip_dense_kernel", "achieved": achieved, "peak": int8_burst,
+                    "unit": "TFLOP/s", "frac": achieved / int8_burst,
+                    "peak_source": "%s bf16 cuBLAS burst x2 (nominal int8:bf16 ratio)" % peaks["_source"],
+                    "frac_of_sustained": achieved / int8_sust, "frac_of_nominal_4500": achieved / NOMINAL_INT8_TOPS,
+                    "traffic": NCU_TRAFFIC_BYTES[args.workload]}
+    else:
+        achieved = args.steps * step_bytes / (kernel_ms * 1e-3) / 1e9
+        kname = "mip_skinny_kernel" if args.workload == "skinny" else "mip_dense_kernel"
+        roofline = {"bound": "hbm", "kernel": kname, "achieved": achieved, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                    "peak_source": "%s copy bandwidth" % peaks["_source"],
+                    "traffic": NCU_TRAFFIC_BYTES[args.workload]}
+    roofline["launches_timed"] = n_launch
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
+    e2e = None
+    if args.workload == "square" and not args.no_e2e:
+        pinned = []
+        for p in probs:
+            n = p.dims[0]
+            hA = torch.from_numpy(p.host[0].view(np.uint8)).pin_memory()
+            hB = torch.from_numpy(p.host[1].view(np.uint8)).pin_memory()
+            hC = torch.empty(n * n, dtype=torch.int32).pin_memory()
+            pinned.append((n, hA, hB, hC))
+        h2d = sum(2 * n * n for (n, _a, _b, _c) in pinned)
+        d2h = sum(4 * n * n for (n, _a, _b, _c) in pinned)
+
+        def e2e_step():
+            for (n, hA, hB, hC) in pinned:
+                mg.mipgemm_host_s8s8s32(n, n, n, hA, n, hB, n, hC, n, 0)
+
+        e2e_step()
+        e2e_steps = max(1, min(args.steps, 3))
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_step()
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0) / e2e_steps
+        e2e = {"value": world * step_ops / e2e_s / 1e12, "unit": "TOPS", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "steps": e2e_steps,
+               "api": "mipgemm_host_s8s8s32 (pinned host buffers, cudaMemcpy2DAsync both ways)"}
+        del pinned
+
+    # ---- the CPU oracle on a bounded sample of the same workload, same run
+    cpu = None
+    if want_cpu:
+        from oracle import mip_oracle as orc
+        frac = calibrate_fraction(probs, 15.0)
+        gpu_rows = {}
+        for p, r in zip(probs, oracle_sample_rows(probs, frac)):
+            n = p.dims[1]
+            gpu_rows[p.name] = p.bufs[2][:r * n].cpu().numpy()
+        secs, ops, parity = time_oracle_sample(probs, frac, compare_with=gpu_rows)
+        rows = oracle_sample_rows(probs, frac)
+        cpu = {"value": ops / secs / 1e12, "unit": "TOPS", "cores": orc.threads(), "kind": "oracle",
+               "sample": "first rows of every sweep member (%s), %.1f s of CPU time" % (
+                   ", ".join("%d/%d" % (r, p.dims[0]) for r, p in zip(rows, probs)), secs),
+               "gpu_rows_match_oracle": parity}
+
+    line = {
+        "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": workload,
+                   "l2": "operands + outputs of one step exceed the 126 MB L2 many times over; "
+                         "every buffer is evicted between two uses",
+                   "launches_per_step": len(order)},
+        "clocks": sampler.summary(),
+        "e2e": e2e,
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+    }
+    if args.detail:
+        line["per_problem"] = detail
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -125,7 +125,25 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
                          const uint8_t *X, const int8_t *Wt, int32_t *Y,
                          int accumulate, void *stream);
 
+/*
+ * Host-buffer variants (the end-to-end path): A, B and C are HOST pointers (pinned or
+ * pageable) with the same layouts as above.  The call stages the operands into device
+ * memory obtained with cudaMallocAsync on `stream`, runs the device entry point, copies
+ * the M x N result back into C (padding columns of the host C are left untouched; with
+ * accumulate != 0 the host C is uploaded first), releases the device memory and
+ * SYNCHRONISES the stream before returning.  Same return codes as the device variants.
+ */
+int mipgemm_host_s8s8s32(int64_t M, int64_t N, int64_t K,
+                         const int8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                         int32_t *C, int64_t ldc, int accumulate, void *stream);
+int mipgemm_host_u8s8s32(int64_t M, int64_t N, int64_t K,
+                         const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                         int32_t *C, int64_t ldc, int accumulate, void *stream);
+
 /* ---- support calls (no counterpart in the paper) ---- */
+
+/* Number of kernels this library has enqueued since it was loaded (all threads, all devices). */
+uint64_t mipgemm_launch_count(void);
 
 /* Synchronises `stream` and returns MIPGEMM_OK, MIPGEMM_ERR_TIMEOUT if any kernel
  * since the last call gave up a bounded wait (the flag is then cleared), or

@@ -33,6 +33,9 @@ SIGNATURES = {
     "mipgemm_s8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_u8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_conv_u8s8s32": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, _int, _vp]),
+    "mipgemm_host_s8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
+    "mipgemm_host_u8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
+    "mipgemm_launch_count": (ctypes.c_uint64, []),
     "mipgemm_device_status": (_int, [_vp]),
     "mipgemm_set_workspace": (_int, [_vp, _sz]),
     "mipgemm_workspace_query_gemm": (_sz, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int]),
@@ -98,6 +101,22 @@ def mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, p
     return _check(_lib.mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
                                             dil_h, dil_w, _ptr(X), _ptr(Wt), _ptr(Y),
                                             int(bool(accumulate)), _stream(stream)), check)
+
+
+def mipgemm_host_s8s8s32(M, N, K, A, lda, B, ldb, C, ldc, accumulate=0, stream=None, check=True) -> int:
+    """Host-buffer variant: A, B, C are host tensors/arrays (``data_ptr()``) or raw host addresses;
+    copies in, computes on the device, copies C back and synchronises."""
+    return _check(_lib.mipgemm_host_s8s8s32(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                            int(bool(accumulate)), _stream(stream)), check)
+
+
+def mipgemm_host_u8s8s32(M, N, K, A, lda, B, ldb, C, ldc, accumulate=0, stream=None, check=True) -> int:
+    return _check(_lib.mipgemm_host_u8s8s32(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                            int(bool(accumulate)), _stream(stream)), check)
+
+
+def mipgemm_launch_count() -> int:
+    return int(_lib.mipgemm_launch_count())
 
 
 def mipgemm_device_status(stream=None) -> int:

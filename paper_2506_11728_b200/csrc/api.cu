@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <atomic>
 #include <mutex>
 
 #include "../../include/mipgemm.h"
@@ -20,6 +21,7 @@ struct Tuning {
     int block_n = 0, stages = 0, split_k = 0, force_path = 0;
 };
 Tuning g_tuning;
+std::atomic<uint64_t> g_launches{0};
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -35,6 +37,7 @@ struct DeviceState {
     bool ready = false;
     int status = MIPGEMM_OK;
     int sm_count = 0;
+    int pair_clusters = 0;                 // co-resident 2-CTA clusters of the pair kernel
     unsigned int* status_word = nullptr;   // device
     void* lent = nullptr;
     size_t lent_bytes = 0;
@@ -80,6 +83,7 @@ int get_device(DeviceState** out) {
                 g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(fn);
             }
             if ((e = dense_init()) != cudaSuccess) return cuda_fail(e);
+            d.pair_clusters = dense_pair_max_clusters(kSmemBudget);
             if ((e = cudaMalloc(&d.status_word, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaMemset(d.status_word, 0, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
             d.status = MIPGEMM_OK;
@@ -184,17 +188,28 @@ uint32_t pow2_at_least(uint32_t v) {
 
 // Tile width, pipeline depth and split-K for an M x N x K problem (k-block = block_k bytes).
 struct Plan {
+    int pair;   // 1: CTA pairs share 256-row tiles (cta_group::2)
     int block_n, stages, split_k, kb_per_split, k_blocks, tiles_m, tiles_n;
 };
 
-Plan make_plan(long long M, long long N, long long K, int block_k, int sm_count) {
+Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceState* dev) {
+    const int sm_count = dev->sm_count;
     Plan pl{};
-    pl.tiles_m = static_cast<int>((M + kBlockM - 1) / kBlockM);
     pl.k_blocks = static_cast<int>((K + block_k - 1) / block_k);
+    // CTA pairs pay off when there is at least a full wave of 256 x 256 tiles.
+    const long long pair_tiles = ((M + 2 * kBlockM - 1) / (2 * kBlockM)) * ((N + 255) / 256);
+    pl.pair = (dev->pair_clusters > 0 && pair_tiles >= dev->pair_clusters && !g_tuning.block_n) ? 1 : 0;
+    if (g_tuning.force_path == MIPGEMM_PATH_DENSE_PAIR && dev->pair_clusters > 0) pl.pair = 1;
+    if (g_tuning.force_path == MIPGEMM_PATH_DENSE) pl.pair = 0;
+    const int rows_per_tile = pl.pair ? 2 * kBlockM : kBlockM;
+    pl.tiles_m = static_cast<int>((M + rows_per_tile - 1) / rows_per_tile);
     auto tiles_for = [&](int bn) { return static_cast<long long>(pl.tiles_m) * ((N + bn - 1) / bn); };
     int bn;
     if (g_tuning.block_n) {
         bn = g_tuning.block_n;
+        if (pl.pair && bn % 64 != 0) bn = (bn + 63) / 64 * 64;
+    } else if (pl.pair) {
+        bn = 256;
     } else if (N <= 64) {
         bn = 64;
     } else if (N <= 128) {
@@ -209,7 +224,7 @@ Plan make_plan(long long M, long long N, long long K, int block_k, int sm_count)
     }
     pl.block_n = bn;
     pl.tiles_n = static_cast<int>((N + bn - 1) / bn);
-    const int stage_bytes = kBlockM * block_k + bn * block_k;
+    const int stage_bytes = kBlockM * block_k + (pl.pair ? bn / 2 : bn) * block_k;
     int stages = (kSmemBudget - kCtrlBytes - 1024) / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
     if (g_tuning.stages) stages = g_tuning.stages < stages ? g_tuning.stages : stages;
@@ -219,7 +234,7 @@ Plan make_plan(long long M, long long N, long long K, int block_k, int sm_count)
     const long long tiles = static_cast<long long>(pl.tiles_m) * pl.tiles_n;
     if (g_tuning.split_k) {
         split = g_tuning.split_k;
-    } else if (tiles * 2 <= sm_count && pl.k_blocks >= 8) {
+    } else if (!pl.pair && tiles * 2 <= sm_count && pl.k_blocks >= 8) {
         split = static_cast<int>(sm_count / tiles);
         const int max_split = pl.k_blocks / 4;
         if (split > max_split) split = max_split;
@@ -251,7 +266,8 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
     const uintptr_t c_addr = reinterpret_cast<uintptr_t>(C);
     p.store_vec = (c_addr % 32 == 0 && ldc % 8 == 0) ? 8 : ((c_addr % 16 == 0 && ldc % 4 == 0) ? 4 : 1);
     p.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | (1u << 10) |
-              (static_cast<uint32_t>(pl.block_n >> 3) << 17) | (static_cast<uint32_t>(kBlockM >> 4) << 24);
+              (static_cast<uint32_t>(pl.block_n >> 3) << 17) |
+              (static_cast<uint32_t>((pl.pair ? 2 * kBlockM : kBlockM) >> 4) << 24);
     p.tmem_cols = pow2_at_least(2u * pl.block_n);
     p.a_im2col = 0;
     p.status = dev->status_word;
@@ -262,13 +278,22 @@ int run_dense(DenseParams& p, const Plan& pl, long long M, long long N, int32_t*
               int accumulate, DeviceState* dev, cudaStream_t stream) {
     if (pl.split_k > 1 && !accumulate) {
         cudaError_t e = launch_fill_zero(C, ldc, M, N, stream);
+        ++g_launches;
         if (e != cudaSuccess) return cuda_fail(e);
     }
     const long long units = static_cast<long long>(pl.tiles_m) * pl.tiles_n * pl.split_k;
-    const int grid = static_cast<int>(units < dev->sm_count ? units : dev->sm_count);
-    const size_t smem = static_cast<size_t>(pl.stages) * (kBlockM * p.block_k + pl.block_n * p.block_k) +
+    const int b_rows = pl.pair ? pl.block_n / 2 : pl.block_n;
+    const size_t smem = static_cast<size_t>(pl.stages) * (kBlockM * p.block_k + b_rows * p.block_k) +
                         kCtrlBytes + 1024;
-    cudaError_t e = launch_dense(p, grid, smem, stream);
+    cudaError_t e;
+    if (pl.pair) {
+        const int clusters = static_cast<int>(units < dev->pair_clusters ? units : dev->pair_clusters);
+        e = launch_dense_pair(p, 2 * clusters, smem, stream);
+    } else {
+        const int grid = static_cast<int>(units < dev->sm_count ? units : dev->sm_count);
+        e = launch_dense(p, grid, smem, stream);
+    }
+    ++g_launches;
     if (e != cudaSuccess) return cuda_fail(e);
     return MIPGEMM_OK;
 }
@@ -308,17 +333,19 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
         tl_last_path = MIPGEMM_PATH_TRIVIAL | path_flags;
         if (!accumulate) {
             cudaError_t e = launch_fill_zero(C, ldc, M, N, stream);
+            ++g_launches;
             if (e != cudaSuccess) return cuda_fail(e);
         }
         return MIPGEMM_OK;
     }
 
     // ---- skinny path
-    if (M <= 16 && g_tuning.force_path != MIPGEMM_PATH_DENSE) {
+    if (M <= 16 && g_tuning.force_path != MIPGEMM_PATH_DENSE && g_tuning.force_path != MIPGEMM_PATH_DENSE_PAIR) {
         SkinnyParams sp{A, lda, B, ldb, C, ldc, static_cast<int>(M), static_cast<int>(N),
                         static_cast<int>(K), a_unsigned ? 1 : 0, accumulate ? 1 : 0};
         if (skinny_supported(sp)) {
             cudaError_t e = launch_skinny(sp, stream);
+            ++g_launches;
             if (e != cudaSuccess) return cuda_fail(e);
             tl_last_path = MIPGEMM_PATH_SKINNY | path_flags;
             return MIPGEMM_OK;
@@ -338,6 +365,7 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     if (repack_a) {
         void* dst = scratch.take(static_cast<size_t>(M) * pitch);
         cudaError_t e = launch_repack(A, lda, dst, pitch, M, K, stream);
+        ++g_launches;
         if (e != cudaSuccess) return cuda_fail(e);
         a_use = dst;
         lda_use = pitch;
@@ -346,6 +374,7 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     if (repack_b) {
         void* dst = scratch.take(static_cast<size_t>(N) * pitch);
         cudaError_t e = launch_repack(B, ldb, dst, pitch, N, K, stream);
+        ++g_launches;
         if (e != cudaSuccess) return cuda_fail(e);
         b_use = dst;
         ldb_use = pitch;
@@ -353,15 +382,17 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     }
 
     const int block_k = 128;
-    const Plan pl = make_plan(M, N, K, block_k, dev->sm_count);
+    const Plan pl = make_plan(M, N, K, block_k, dev);
     DenseParams p;
     std::memset(&p, 0, sizeof(p));
     fill_common(p, pl, M, N, C, ldc, block_k, a_unsigned, accumulate, dev);
     if ((st = encode_tiled_2d(&p.tmap_a, a_use, K, M, lda_use, block_k, kBlockM)) != MIPGEMM_OK) return st;
-    if ((st = encode_tiled_2d(&p.tmap_b, b_use, K, N, ldb_use, block_k, pl.block_n)) != MIPGEMM_OK) return st;
+    if ((st = encode_tiled_2d(&p.tmap_b, b_use, K, N, ldb_use, block_k, pl.pair ? pl.block_n / 2 : pl.block_n)) !=
+        MIPGEMM_OK)
+        return st;
     if ((st = run_dense(p, pl, M, N, C, ldc, accumulate, dev, stream)) != MIPGEMM_OK) return st;
     if (pl.split_k > 1) path_flags |= MIPGEMM_PATH_SPLITK;
-    tl_last_path = MIPGEMM_PATH_DENSE | path_flags;
+    tl_last_path = (pl.pair ? MIPGEMM_PATH_DENSE_PAIR : MIPGEMM_PATH_DENSE) | path_flags;
     return MIPGEMM_OK;
 }
 
@@ -394,6 +425,55 @@ bool conv_tma_eligible(const ConvGeom& g, const void* X, const void* Wt) {
     if (g.W >= (1LL << 31) || g.H >= (1LL << 31) || g.Nb >= (1LL << 31)) return false;
     if (g.H * g.W * g.Cin >= (1LL << 40)) return false;
     return true;
+}
+
+// Host-buffer front end: stage operands, run the device entry point, copy C back.
+int host_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, const int8_t* B,
+              int64_t ldb, int32_t* C, int64_t ldc, int accumulate, void* stream_v) {
+    if (M < 0 || N < 0 || K < 0 || lda < K || ldb < K || ldc < N) return MIPGEMM_ERR_INVALID_ARG;
+    if (K > (a_unsigned ? 65793 : 131071)) return MIPGEMM_ERR_K_TOO_LARGE;
+    if (M == 0 || N == 0) return MIPGEMM_OK;
+    if (!C || (K > 0 && (!A || !B))) return MIPGEMM_ERR_INVALID_ARG;
+    DeviceState* dev = nullptr;
+    int st = get_device(&dev);
+    if (st != MIPGEMM_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const long long pitch = round_up(K > 0 ? K : 1, 16);
+    const long long ldc_dev = round_up(N, 8);
+    const size_t a_bytes = align256(static_cast<size_t>(M) * pitch);
+    const size_t b_bytes = align256(static_cast<size_t>(N) * pitch);
+    const size_t c_bytes = align256(static_cast<size_t>(M) * ldc_dev * 4);
+    char* base = nullptr;
+    cudaError_t e = cudaMallocAsync(reinterpret_cast<void**>(&base), a_bytes + b_bytes + c_bytes, stream);
+    if (e != cudaSuccess) {
+        tl_last_cuda_error = static_cast<int>(e);
+        (void)cudaGetLastError();
+        return MIPGEMM_ERR_WORKSPACE;
+    }
+    void* dA = base;
+    void* dB = base + a_bytes;
+    int32_t* dC = reinterpret_cast<int32_t*>(base + a_bytes + b_bytes);
+    st = MIPGEMM_OK;
+    if (K > 0) {
+        e = cudaMemcpy2DAsync(dA, pitch, A, lda, K, M, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaMemcpy2DAsync(dB, pitch, B, ldb, K, N, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) st = cuda_fail(e);
+    }
+    if (st == MIPGEMM_OK && accumulate) {
+        e = cudaMemcpy2DAsync(dC, ldc_dev * 4, C, ldc * 4, N * 4, M, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) st = cuda_fail(e);
+    }
+    if (st == MIPGEMM_OK)
+        st = gemm_impl(a_unsigned, M, N, K, dA, pitch, static_cast<const int8_t*>(dB), pitch, dC, ldc_dev,
+                       accumulate, stream_v, 0);
+    if (st == MIPGEMM_OK) {
+        e = cudaMemcpy2DAsync(C, ldc * 4, dC, ldc_dev * 4, N * 4, M, cudaMemcpyDeviceToHost, stream);
+        if (e != cudaSuccess) st = cuda_fail(e);
+    }
+    (void)cudaFreeAsync(base, stream);
+    e = cudaStreamSynchronize(stream);
+    if (st == MIPGEMM_OK && e != cudaSuccess) st = cuda_fail(e);
+    return st;
 }
 
 }  // namespace
@@ -436,7 +516,7 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
 
     if (conv_tma_eligible(g, X, Wt) && g_tuning.force_path != MIPGEMM_PATH_IM2COL_EXPLICIT) {
         const int block_k = (Cin % 128 == 0) ? 128 : 64;
-        const Plan pl = make_plan(M, Cout, K, block_k, dev->sm_count);
+        const Plan pl = make_plan(M, Cout, K, block_k, dev);
         DenseParams p;
         std::memset(&p, 0, sizeof(p));
         fill_common(p, pl, M, Cout, Y, Cout, block_k, true, accumulate, dev);
@@ -449,9 +529,12 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
         p.pad_w = pad_w; p.pad_h = pad_h;
         p.dil_w = dil_w; p.dil_h = dil_h;
         if ((st = encode_im2col(&p.tmap_a, X, g, block_k, kBlockM)) != MIPGEMM_OK) return st;
-        if ((st = encode_tiled_2d(&p.tmap_b, Wt, K, Cout, K, block_k, pl.block_n)) != MIPGEMM_OK) return st;
+        if ((st = encode_tiled_2d(&p.tmap_b, Wt, K, Cout, K, block_k, pl.pair ? pl.block_n / 2 : pl.block_n)) !=
+            MIPGEMM_OK)
+            return st;
         if ((st = run_dense(p, pl, M, Cout, Y, Cout, accumulate, dev, stream)) != MIPGEMM_OK) return st;
-        tl_last_path = MIPGEMM_PATH_DENSE | MIPGEMM_PATH_IM2COL_TMA | (pl.split_k > 1 ? MIPGEMM_PATH_SPLITK : 0);
+        tl_last_path = (pl.pair ? MIPGEMM_PATH_DENSE_PAIR : MIPGEMM_PATH_DENSE) | MIPGEMM_PATH_IM2COL_TMA |
+                       (pl.split_k > 1 ? MIPGEMM_PATH_SPLITK : 0);
         return MIPGEMM_OK;
     }
 
@@ -466,6 +549,7 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
     Im2colParams ip{X, cols, g.Nb, g.H, g.W, g.Cin, g.Ho, g.Wo, R, S, stride_h, stride_w,
                     pad_h, pad_w, dil_h, dil_w, K, k_pitch};
     cudaError_t e = launch_im2col(ip, stream);
+    ++g_launches;
     if (e != cudaSuccess) return cuda_fail(e);
     // The GEMM takes its own share (weight re-pitching when K % 16 != 0) from the same lease.
     return gemm_impl(true, M, Cout, K, cols, k_pitch, Wt, K, Y, Cout, accumulate, stream_v,
@@ -520,6 +604,18 @@ size_t mipgemm_workspace_query_conv(int64_t Nb, int64_t H, int64_t W, int64_t Ci
     return align256(static_cast<size_t>(M) * k_pitch) + gemm_scratch_bytes(M, Cout, K, nullptr, k_pitch, nullptr, K);
 }
 
+int mipgemm_host_s8s8s32(int64_t M, int64_t N, int64_t K, const int8_t* A, int64_t lda, const int8_t* B,
+                         int64_t ldb, int32_t* C, int64_t ldc, int accumulate, void* stream) {
+    return host_impl(false, M, N, K, A, lda, B, ldb, C, ldc, accumulate, stream);
+}
+
+int mipgemm_host_u8s8s32(int64_t M, int64_t N, int64_t K, const uint8_t* A, int64_t lda, const int8_t* B,
+                         int64_t ldb, int32_t* C, int64_t ldc, int accumulate, void* stream) {
+    return host_impl(true, M, N, K, A, lda, B, ldb, C, ldc, accumulate, stream);
+}
+
+uint64_t mipgemm_launch_count(void) { return g_launches.load(); }
+
 int mipgemm_last_path(void) { return tl_last_path; }
 int mipgemm_last_cuda_error(void) { return tl_last_cuda_error; }
 
@@ -545,6 +641,7 @@ int mipgemm_probe_i8_peak(int iters, int* grid_out, double* ops_per_launch, int3
     if (st != MIPGEMM_OK) return st;
     const int grid = dev->sm_count;
     cudaError_t e = launch_probe(iters, grid, sink, static_cast<cudaStream_t>(stream_v));
+    ++g_launches;
     if (e != cudaSuccess) return cuda_fail(e);
     if (grid_out) *grid_out = grid;
     if (ops_per_launch) *ops_per_launch = 2.0 * 128 * 256 * 128 * static_cast<double>(iters) * grid;

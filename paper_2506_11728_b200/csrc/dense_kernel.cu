@@ -7,13 +7,22 @@
 // memory, loops L1-L5 become a persistent tile scheduler, and the load/store of
 // C_r becomes the epilogue that drains tensor memory to global memory.
 //
-// One CTA = 6 warps: warp 0 lane 0 issues TMA loads, warp 1 lane 0 issues MMAs
-// (warp 1 also owns the tensor-memory allocation), warps 2-5 are the epilogue
+// One CTA = 6 warps: warp 0 issues TMA loads, warp 1 issues MMAs (one elected lane
+// each; warp 1 also owns the tensor-memory allocation), warps 2-5 are the epilogue
 // (warp w reads TMEM lanes 32*(w%4) .. +31).  Two accumulators alternate so the
 // epilogue of tile t overlaps the main loop of tile t+1.  Every wait is bounded;
 // on expiry the CTA raises an abort word, all roles unwind, outstanding copies
 // and MMAs are drained with a bounded wait, tensor memory is released and bit 0
 // of *status is set.
+//
+// The kernel exists in two forms.  kPair = false: one CTA per 128 x block_n tile
+// (cta_group::1).  kPair = true: clusters of two CTAs share a 256 x block_n tile
+// (cta_group::2): each CTA stages its own 128 rows of A and HALF of the B tile, the
+// leader CTA (cluster rank 0) issues every MMA, and both CTAs' tensor memories receive
+// their 128 rows of the accumulator -- B traffic from L2 and shared memory is halved.
+// Both CTAs' TMA loads complete on the leader's "full" barrier; MMA completion is
+// committed to each CTA's own "empty" / "tmem_full" barrier with two plain commits (no
+// multicast form is used anywhere in this file).
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -81,8 +90,16 @@ __device__ __forceinline__ void store_chunk(const DenseParams& p, int32_t* dst, 
     }
 }
 
+template <bool kPair>
 __global__ void __launch_bounds__(kDenseThreads, 1)
 mip_dense_kernel(const __grid_constant__ DenseParams p) {
+    constexpr int kGroup = kPair ? 2 : 1;
+    constexpr int kRowsPerTile = kPair ? 2 * kBlockM : kBlockM;
+    const uint32_t cta_rank = kPair ? cluster_ctarank() : 0u;
+    const bool leader = cta_rank == 0;
+    const int first_unit = kPair ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+    const int unit_stride = kPair ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+    const int b_rows = kPair ? (p.block_n >> 1) : p.block_n;   // rows of B staged by this CTA
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
@@ -90,7 +107,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
     const uint32_t smem_base = raw_addr + pad;
 
     const uint32_t a_bytes = kBlockM * p.block_k;
-    const uint32_t b_bytes = p.block_n * p.block_k;
+    const uint32_t b_bytes = b_rows * p.block_k;
     const uint32_t stage_bytes = a_bytes + b_bytes;
     const uint32_t ctrl = smem_base + p.stages * stage_bytes;
     // control block: full[stages] | empty[stages] | tmem_full[2] | tmem_empty[2] | drain | slot | abort
@@ -103,7 +120,10 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl_ptr + 16 * p.stages + 40);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
 
-    const int warp = threadIdx.x >> 5;
+    // Broadcasting the warp index makes it provably warp-uniform for the compiler, so each
+    // role's loop runs convergently (addresses, counters and descriptors live in uniform
+    // registers) and only the single-thread instructions are issued under elect_one().
+    const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0);
     const int lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -113,7 +133,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull + 8u * a, 1);
-            mbar_init(bar_tempty + 8u * a, 4);
+            mbar_init(bar_tempty + 8u * a, kPair ? 8 : 4);
         }
         mbar_init(bar_drain, 1);
         *abort_flag = 0;
@@ -122,11 +142,15 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         tma_prefetch_desc(&p.tmap_b);
     }
     if (warp == 1) {
-        tmem_alloc<1>(smem_u32(tmem_slot), p.tmem_cols);
-        tmem_relinquish<1>();
+        tmem_alloc<kGroup>(smem_u32(tmem_slot), p.tmem_cols);
+        tmem_relinquish<kGroup>();
     }
     tc_fence_before();
     __syncthreads();
+    if (kPair) {   // the peer's barriers must be initialised before anything remote touches them
+        cluster_arrive();
+        cluster_wait();
+    }
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -134,67 +158,94 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
     const uint64_t budget = p.wait_budget_ns;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            uint32_t s = 0, phase = 0, issued = 0;
-            bool ok = true;
-            for (int unit = blockIdx.x; unit < total_units && ok; unit += gridDim.x) {
-                const TileCoord tc = decode_unit(p, unit, kBlockM);
-                int cw = 0, chh = 0, cn = 0;
-                if (p.a_im2col) {
-                    cn = tc.m0 / p.conv_howo;
-                    const int rem = tc.m0 - cn * p.conv_howo;
-                    const int ho = rem / p.conv_wo;
-                    const int wo = rem - ho * p.conv_wo;
-                    cw = wo * p.stride_w - p.pad_w;
-                    chh = ho * p.stride_h - p.pad_h;
-                }
-                for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb) {
-                    if (!mbar_wait(bar_empty + 8u * s, phase ^ 1u, abort_flag, budget)) { ok = false; break; }
-                    const uint32_t full = bar_full + 8u * s;
-                    const uint32_t a_dst = smem_base + s * stage_bytes;
-                    mbar_arrive_expect_tx(full, stage_bytes);
-                    if (p.a_im2col) {
-                        const int tap = kb / p.c_chunks;
-                        const int cc = kb - tap * p.c_chunks;
-                        const int fr = tap / p.conv_s;
-                        const int fs = tap - fr * p.conv_s;
-                        tma_load_im2col_4d(a_dst, &p.tmap_a, full, cc * p.block_k, cw, chh, cn,
-                                           static_cast<uint16_t>(fs * p.dil_w),
-                                           static_cast<uint16_t>(fr * p.dil_h));
-                    } else {
-                        tma_load_2d(a_dst, &p.tmap_a, full, kb * p.block_k, tc.m0);
-                    }
-                    tma_load_2d(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, tc.n0);
-                    ++issued;
-                    if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
-                }
+        // ------------------------------------------------------------ TMA producer (whole warp loops)
+        uint32_t s = 0, phase = 0, issued = 0;
+        bool ok = true;
+        const uint32_t tx_bytes = kPair ? 2u * stage_bytes : stage_bytes;
+        for (int unit = first_unit; unit < total_units && ok; unit += unit_stride) {
+            const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
+            const int m_cta = tc.m0 + static_cast<int>(cta_rank) * kBlockM;
+            const int n_cta = tc.n0 + static_cast<int>(cta_rank) * b_rows;
+            int cw = 0, chh = 0, cn = 0;
+            if (p.a_im2col) {
+                // a peer CTA whose rows all lie beyond M gathers from pixel 0 instead (its
+                // accumulator rows are never stored)
+                const int m_src = m_cta < p.M ? m_cta : 0;
+                cn = m_src / p.conv_howo;
+                const int rem = m_src - cn * p.conv_howo;
+                const int ho = rem / p.conv_wo;
+                const int wo = rem - ho * p.conv_wo;
+                cw = wo * p.stride_w - p.pad_w;
+                chh = ho * p.stride_h - p.pad_h;
             }
-            if (!ok) {
-                // Unwinding: wait (bounded) until every copy already issued has landed.
-                const uint32_t n = min(issued, static_cast<uint32_t>(p.stages));
-                for (uint32_t i = 1; i <= n; ++i) {
-                    const uint32_t idx = issued - i;
-                    const uint32_t st = idx % p.stages;
-                    const uint32_t ph = (idx / p.stages) & 1u;
-                    const uint64_t t0 = globaltimer_ns();
-                    while (!mbar_try_wait(bar_full + 8u * st, ph)) {
-                        if (globaltimer_ns() - t0 > budget) break;
+            int tap = 0, cc = 0, fr = 0, fs = 0;
+            if (p.a_im2col) {
+                tap = tc.kb_begin / p.c_chunks;
+                cc = tc.kb_begin - tap * p.c_chunks;
+                fr = tap / p.conv_s;
+                fs = tap - fr * p.conv_s;
+            }
+            for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb) {
+                if (!mbar_wait(bar_empty + 8u * s, phase ^ 1u, abort_flag, budget)) { ok = false; break; }
+                // both CTAs' bytes complete on the leader's barrier, which expects all of them
+                const uint32_t full_local = bar_full + 8u * s;
+                const uint32_t full = kPair ? mapa_u32(full_local, 0) : full_local;
+                const uint32_t a_dst = smem_base + s * stage_bytes;
+                if (elect_one()) {
+                    if (leader) mbar_arrive_expect_tx(full_local, tx_bytes);
+                    if (p.a_im2col) {
+                        if (kPair)
+                            tma_load_im2col_4d_pair(a_dst, &p.tmap_a, full, cc * p.block_k, cw, chh, cn,
+                                                    static_cast<uint16_t>(fs * p.dil_w),
+                                                    static_cast<uint16_t>(fr * p.dil_h));
+                        else
+                            tma_load_im2col_4d(a_dst, &p.tmap_a, full, cc * p.block_k, cw, chh, cn,
+                                               static_cast<uint16_t>(fs * p.dil_w),
+                                               static_cast<uint16_t>(fr * p.dil_h));
+                    } else if (kPair) {
+                        tma_load_2d_pair(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta);
+                    } else {
+                        tma_load_2d(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta);
                     }
+                    if (kPair)
+                        tma_load_2d_pair(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta);
+                    else
+                        tma_load_2d(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta);
+                }
+                if (p.a_im2col && ++cc == p.c_chunks) {   // next filter tap (r, s)
+                    cc = 0;
+                    if (++fs == p.conv_s) { fs = 0; ++fr; }
+                }
+                ++issued;
+                if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
+            }
+        }
+        if (!ok && leader) {
+            // Unwinding: wait (bounded) until every copy already issued has landed.  (A peer
+            // CTA cannot observe its copies -- they complete on the leader's barrier; it is
+            // held by the final cluster barrier until the leader has finished unwinding.)
+            const uint32_t n = min(issued, static_cast<uint32_t>(p.stages));
+            for (uint32_t i = 1; i <= n; ++i) {
+                const uint32_t idx = issued - i;
+                const uint32_t st = idx % p.stages;
+                const uint32_t ph = (idx / p.stages) & 1u;
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(bar_full + 8u * st, ph)) {
+                    if (globaltimer_ns() - t0 > budget) break;
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuer (whole warp loops)
+        if (leader) {
             uint32_t s = 0, phase = 0;
             const uint32_t k_steps = p.block_k / 32;
             bool ok = true;
             int t = 0;
-            for (int unit = blockIdx.x; unit < total_units && ok; unit += gridDim.x, ++t) {
-                const TileCoord tc = decode_unit(p, unit, kBlockM);
+            for (int unit = first_unit; unit < total_units && ok; unit += unit_stride, ++t) {
+                const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
                 const uint32_t acc = t & 1, acc_phase = (t >> 1) & 1;
-                if (!mbar_wait(bar_tempty + 8u * acc, acc_phase ^ 1u, abort_flag, budget)) { ok = false; break; }
+                if (!mbar_wait<kPair>(bar_tempty + 8u * acc, acc_phase ^ 1u, abort_flag, budget)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * p.block_n;
                 for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb) {
@@ -203,18 +254,40 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     const uint32_t a_addr = smem_base + s * stage_bytes;
                     const uint64_t a_desc = make_kmajor_desc(a_addr, p.block_k);
                     const uint64_t b_desc = make_kmajor_desc(a_addr + a_bytes, p.block_k);
-                    for (uint32_t k = 0; k < k_steps; ++k) {
-                        mma_i8<1>(d_tmem, a_desc + 2ull * k, b_desc + 2ull * k, p.idesc,
-                                  (kb > tc.kb_begin || k > 0) ? 1u : 0u);
+                    const uint32_t empty_local = bar_empty + 8u * s;
+                    const uint32_t empty_peer = kPair ? mapa_u32(empty_local, 1) : 0u;
+                    if (elect_one()) {
+                        for (uint32_t k = 0; k < k_steps; ++k) {
+                            mma_i8<kGroup>(d_tmem, a_desc + 2ull * k, b_desc + 2ull * k, p.idesc,
+                                           (kb > tc.kb_begin || k > 0) ? 1u : 0u);
+                        }
+                        if (kPair) {
+                            mma_commit_pair(empty_local);
+                            mma_commit_pair(empty_peer);
+                        } else {
+                            mma_commit(empty_local);
+                        }
                     }
-                    mma_commit(bar_empty + 8u * s);
                     if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
                 }
-                if (ok) mma_commit(bar_tfull + 8u * acc);
+                if (ok) {
+                    const uint32_t tfull_local = bar_tfull + 8u * acc;
+                    const uint32_t tfull_peer = kPair ? mapa_u32(tfull_local, 1) : 0u;
+                    if (elect_one()) {
+                        if (kPair) {
+                            mma_commit_pair(tfull_local);
+                            mma_commit_pair(tfull_peer);
+                        } else {
+                            mma_commit(tfull_local);
+                        }
+                    }
+                }
             }
             if (!ok) {
                 // Unwinding: let every MMA already issued retire before TMEM is released.
-                mma_commit(bar_drain);
+                if (elect_one()) {
+                    if (kPair) mma_commit_pair(bar_drain); else mma_commit(bar_drain);
+                }
                 const uint64_t t0 = globaltimer_ns();
                 while (!mbar_try_wait(bar_drain, 0)) {
                     if (globaltimer_ns() - t0 > budget) break;
@@ -225,15 +298,16 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;
         int t = 0;
-        for (int unit = blockIdx.x; unit < total_units; unit += gridDim.x, ++t) {
-            const TileCoord tc = decode_unit(p, unit, kBlockM);
+        for (int unit = first_unit; unit < total_units; unit += unit_stride, ++t) {
+            const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
             const uint32_t acc = t & 1, acc_phase = (t >> 1) & 1;
             if (!mbar_wait(bar_tfull + 8u * acc, acc_phase, abort_flag, budget)) break;
             tc_fence_after();
-            const int row = tc.m0 + q * 32 + lane;
+            const int m_cta = tc.m0 + static_cast<int>(cta_rank) * kBlockM;
+            const int row = m_cta + q * 32 + lane;
             const int n_rem = p.N - tc.n0;
             const int n_here = min(p.block_n, n_rem);
-            if (tc.m0 + q * 32 < p.M) {
+            if (m_cta + q * 32 < p.M) {
                 int32_t* crow = p.C + static_cast<long long>(row) * p.ldc + tc.n0;
                 const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.block_n;
                 for (int c0 = 0; c0 < n_here; c0 += 32) {
@@ -245,26 +319,75 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty + 8u * acc);
+            if (lane == 0) {
+                if (kPair && !leader) mbar_arrive_remote(bar_tempty + 8u * acc, 0);
+                else mbar_arrive(bar_tempty + 8u * acc);
+            }
         }
     }
 
     tc_fence_before();
     __syncthreads();
+    if (kPair) {   // neither CTA may leave while the other can still reach its shared memory
+        cluster_arrive();
+        cluster_wait();
+    }
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc<1>(tmem_base, p.tmem_cols);
+        tmem_dealloc<kGroup>(tmem_base, p.tmem_cols);
     }
     if (threadIdx.x == 0 && *abort_flag != 0) atomicOr(p.status, 1u);
 }
 
 cudaError_t dense_init() {
-    return cudaFuncSetAttribute(mip_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    cudaError_t e = cudaFuncSetAttribute(mip_dense_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kSmemBudget);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(mip_dense_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                kSmemBudget);
 }
 
 cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream) {
-    mip_dense_kernel<<<grid, kDenseThreads, smem_bytes, stream>>>(p);
+    mip_dense_kernel<false><<<grid, kDenseThreads, smem_bytes, stream>>>(p);
     return cudaGetLastError();
+}
+
+// `grid` counts CTAs and must be even: consecutive CTAs form a cluster of two.
+cudaError_t launch_dense_pair(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+    cfg.blockDim = dim3(kDenseThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true>, p);
+}
+
+// Largest number of co-resident 2-CTA clusters for the pair kernel (0 on failure).
+int dense_pair_max_clusters(size_t smem_bytes) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2, 1, 1);
+    cfg.blockDim = dim3(kDenseThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, mip_dense_kernel<true>, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    return n;
 }
 
 }  // namespace mip

@@ -42,6 +42,7 @@ struct alignas(64) DenseParams {
 
 cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream);
 cudaError_t launch_dense_pair(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream);
+int dense_pair_max_clusters(size_t smem_bytes);
 cudaError_t dense_init();  // opt in to large dynamic shared memory (once per device)
 
 // Skinny-M streaming kernel (M <= 16).
