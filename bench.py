@@ -302,7 +302,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="square", choices=["square", "bert", "resnet", "skinny"])
@@ -311,6 +311,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--detail", action="store_true", help="print per-problem timings to stderr")
+    ap.add_argument("--eager", action="store_true", help="plain launches instead of CUDA-graph replay")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -354,55 +355,96 @@ def main():
             inputs.SKINNY_M, inputs.SKINNY_WEIGHTS)
         unit, metric = "GB/s", "skinny_gemm_gbs"
 
-    # launch order of one step: every problem once (resnet: layer multiplicity; skinny: all slots)
-    order = []
+    # launch order of one step: every problem once (resnet: layer multiplicity; skinny: all
+    # rotation slots), grouped per problem so one event pair brackets each group
+    groups = []
     for p in probs:
         reps = getattr(p, "count", 1) if args.workload == "resnet" else len(p.calls)
-        order.extend([(p, i) for i in range(reps)])
+        groups.append((p, reps))
+    launches_per_step = sum(r for (_p, r) in groups)
 
     def one_step(events=None):
-        for j, (p, i) in enumerate(order):
+        for j, (p, reps) in enumerate(groups):
             if events is not None:
                 events[j][0].record()
-            p.launch(i)
+            for i in range(reps):
+                p.launch(i)
             if events is not None:
                 events[j][1].record()
 
-    stream = torch.cuda.current_stream()
     for _ in range(args.warmup):
         one_step()
     torch.cuda.synchronize()
     assert mg.mipgemm_device_status() == mg.OK
 
+    # One step is captured once as a CUDA graph (kernel launches plus one external timing
+    # event pair per problem) and replayed: the timed region then measures the device, not
+    # the Python interpreter.  --eager times plain launches instead.
+    graph = None
+    count0 = mg.mipgemm_launch_count()
+    if not args.eager:
+        graph_events = [(torch.cuda.Event(enable_timing=True, external=True),
+                         torch.cuda.Event(enable_timing=True, external=True)) for _ in groups]
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            one_step(graph_events)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert mg.mipgemm_device_status() == mg.OK
+    kernels_per_step = (mg.mipgemm_launch_count() - count0) if graph is not None else None
+
     # ---- timed region: exactly K steps between two synchronisation points
-    per_launch = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                   for _ in order] for _ in range(args.steps)]
     sampler = ClockSampler(torch, local_rank)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     launches0 = mg.mipgemm_launch_count()
     sampler.start()
+    stream = torch.cuda.current_stream()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record(stream)
-    for s in range(args.steps):
-        one_step(per_launch[s])
-    ev1.record(stream)
-    torch.cuda.synchronize()
+    group_ms = [0.0] * len(groups)
+    if graph is not None:
+        # the per-problem events are re-recorded by every replay, so they are read after a
+        # separate replay below; the K timed replays run back to back
+        ev0.record(stream)
+        for s in range(args.steps):
+            graph.replay()
+        ev1.record(stream)
+        torch.cuda.synchronize()
+    else:
+        eager_events = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                         for _ in groups] for _ in range(args.steps)]
+        ev0.record(stream)
+        for s in range(args.steps):
+            one_step(eager_events[s])
+        ev1.record(stream)
+        torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    sampler.stop_flag.set()
-    sampler.join(timeout=2.0)
-    launches = mg.mipgemm_launch_count() - launches0
+    launches = (kernels_per_step * args.steps) if graph is not None else (mg.mipgemm_launch_count() - launches0)
     assert mg.mipgemm_device_status() == mg.OK
     elapsed_ms = ev0.elapsed_time(ev1)
+    # per-problem durations (still inside the clock-sampled region)
+    detail_reps = 3 if graph is not None else args.steps
+    if graph is not None:
+        for _ in range(detail_reps):
+            graph.replay()
+            torch.cuda.synchronize()
+            for j, (a, b) in enumerate(graph_events):
+                group_ms[j] += a.elapsed_time(b)
+    else:
+        for s in range(args.steps):
+            for j, (a, b) in enumerate(eager_events[s]):
+                group_ms[j] += a.elapsed_time(b)
+    sampler.stop_flag.set()
+    sampler.join(timeout=2.0)
     if world > 1:
         t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         elapsed_ms = float(t.item())
 
-    step_ops = sum(p.ops for (p, _i) in order)
-    step_bytes = sum(p.bytes for (p, _i) in order)
+    step_ops = sum(p.ops * r for (p, r) in groups)
+    step_bytes = sum(p.bytes * r for (p, r) in groups)
     ms_per_step = elapsed_ms / args.steps
     if unit == "TOPS":
         value = world * step_ops / (ms_per_step * 1e-3) / 1e12
@@ -410,26 +452,21 @@ def main():
         value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
 
     # ---- per-problem kernel time from the events recorded inside the timed region
-    agg = {}
-    for s in range(args.steps):
-        for j, (p, _i) in enumerate(order):
-            a, b = per_launch[s][j]
-            d = agg.setdefault(p.name, [0.0, 0, p])
-            d[0] += a.elapsed_time(b)
-            d[1] += 1
     detail = []
-    for name, (ms, n, p) in agg.items():
-        avg = ms / n
-        detail.append({"name": name, "us": avg * 1e3, "tops": p.ops / (avg * 1e-3) / 1e12,
-                       "gbs": p.bytes / (avg * 1e-3) / 1e9})
+    for j, (p, reps) in enumerate(groups):
+        avg = group_ms[j] / (detail_reps * reps)          # ms per launch of this problem
+        detail.append({"name": p.name, "launches": reps, "us": avg * 1e3,
+                       "tops": p.ops / (avg * 1e-3) / 1e12, "gbs": p.bytes / (avg * 1e-3) / 1e9})
     if args.detail and rank == 0:
         for d in detail:
             sys.stderr.write("%-40s %10.1f us %9.1f TOPS %9.1f GB/s\n" % (d["name"], d["us"], d["tops"], d["gbs"]))
 
     # ---- roofline of the dominant kernel over the timed region
     peaks = load_peaks()
-    kernel_ms = sum(v[0] for v in agg.values())
-    n_launch = sum(v[1] for v in agg.values())
+    # the timed region holds nothing but this workload's kernels, so the dominant kernel's
+    # average launch duration is the region's elapsed time over its launches
+    kernel_ms = elapsed_ms
+    n_launch = launches_per_step * args.steps
     if unit == "TOPS" and args.workload in ("square", "bert"):
         int8_burst = peaks["bf16_tflops"] * (NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS)
         int8_sust = peaks["bf16_tflops_sustained"] * (NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS)
@@ -506,7 +543,8 @@ def main():
         "config": {"workload": workload,
                    "l2": "operands + outputs of one step exceed the 126 MB L2 many times over; "
                          "every buffer is evicted between two uses",
-                   "launches_per_step": len(order)},
+                   "launches_per_step": launches_per_step,
+                   "launch": "eager" if graph is None else "one CUDA graph replay per step"},
         "clocks": sampler.summary(),
         "e2e": e2e,
         "gpu_launches": int(launches),

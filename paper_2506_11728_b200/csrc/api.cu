@@ -21,6 +21,7 @@ struct Tuning {
     int block_n = 0, stages = 0, split_k = 0, force_path = 0;
 };
 Tuning g_tuning;
+bool g_tuning_no_tma_store = false;   // MIPGEMM_DIRECT_STORE=1: force the direct-store epilogue
 std::atomic<uint64_t> g_launches{0};
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -84,6 +85,7 @@ int get_device(DeviceState** out) {
             }
             if ((e = dense_init()) != cudaSuccess) return cuda_fail(e);
             d.pair_clusters = dense_pair_max_clusters(kSmemBudget);
+            if (const char* ds = std::getenv("MIPGEMM_DIRECT_STORE")) g_tuning_no_tma_store = std::atoi(ds) != 0;
             if ((e = cudaMalloc(&d.status_word, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaMemset(d.status_word, 0, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
             d.status = MIPGEMM_OK;
@@ -225,7 +227,7 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
     pl.block_n = bn;
     pl.tiles_n = static_cast<int>((N + bn - 1) / bn);
     const int stage_bytes = kBlockM * block_k + (pl.pair ? bn / 2 : bn) * block_k;
-    int stages = (kSmemBudget - kCtrlBytes - 1024) / stage_bytes;
+    int stages = (kSmemBudget - kCtrlBytes - kStagingBytes - 1024) / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
     if (g_tuning.stages) stages = g_tuning.stages < stages ? g_tuning.stages : stages;
     if (stages < 2) stages = 2;
@@ -269,9 +271,26 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
               (static_cast<uint32_t>(pl.block_n >> 3) << 17) |
               (static_cast<uint32_t>((pl.pair ? 2 * kBlockM : kBlockM) >> 4) << 24);
     p.tmem_cols = pow2_at_least(2u * pl.block_n);
+    // With a 16-byte aligned C (base and pitch) the epilogue writes fully coalesced rows through
+    // shared memory, and split-K partial tiles are added into C by TMA tile reduce-adds.
+    p.c_mode = 0;
+    if (c_addr % 16 == 0 && ldc % 4 == 0 && !g_tuning_no_tma_store) {
+        if (pl.split_k > 1) {
+            p.c_mode = 2;
+            p.use_red = 0;
+        } else {
+            p.c_mode = accumulate ? 3 : 1;
+            if (const char* cm = std::getenv("MIPGEMM_CMODE")) p.c_mode = std::atoi(cm);
+        }
+    }
     p.a_im2col = 0;
     p.status = dev->status_word;
     p.wait_budget_ns = 4000000000ull;
+    p.trace = nullptr;
+#ifdef MIPGEMM_TRACE
+    if (const char* tr = std::getenv("MIPGEMM_TRACE_PTR"))
+        p.trace = reinterpret_cast<unsigned long long*>(std::strtoull(tr, nullptr, 10));
+#endif
 }
 
 int run_dense(DenseParams& p, const Plan& pl, long long M, long long N, int32_t* C, long long ldc,
@@ -284,7 +303,20 @@ int run_dense(DenseParams& p, const Plan& pl, long long M, long long N, int32_t*
     const long long units = static_cast<long long>(pl.tiles_m) * pl.tiles_n * pl.split_k;
     const int b_rows = pl.pair ? pl.block_n / 2 : pl.block_n;
     const size_t smem = static_cast<size_t>(pl.stages) * (kBlockM * p.block_k + b_rows * p.block_k) +
-                        kCtrlBytes + 1024;
+                        kStagingBytes + kCtrlBytes + 1024;
+    if (p.c_mode == 1 || p.c_mode == 2) {
+        cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(M)};
+        cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldc) * 4};
+        cuuint32_t box[2] = {32, static_cast<cuuint32_t>(p.c_mode == 1 ? 128 : 32)};
+        cuuint32_t estr[2] = {1, 1};
+        CUresult r = g_encode_tiled(&p.tmap_c, CU_TENSOR_MAP_DATA_TYPE_INT32, 2, C, dims, strides, box, estr,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            tl_last_cuda_error = 100000 + static_cast<int>(r);
+            return MIPGEMM_ERR_CUDA;
+        }
+    }
     cudaError_t e;
     if (pl.pair) {
         const int clusters = static_cast<int>(units < dev->pair_clusters ? units : dev->pair_clusters);

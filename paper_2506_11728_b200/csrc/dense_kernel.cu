@@ -28,6 +28,15 @@
 
 namespace mip {
 
+#ifdef MIPGEMM_TRACE
+#define MIP_STAMP(slot) do { if (p.trace && blockIdx.x == 0 && (threadIdx.x & 31) == 0) p.trace[slot] = globaltimer_ns(); } while (0)
+__shared__ long long mip_trace_smem[32];
+#define MIP_CLK(slot) do { if (blockIdx.x == 0 && threadIdx.x == 64 && mip_trace_smem[slot] == 0) mip_trace_smem[slot] = clock64(); } while (0)
+#else
+#define MIP_CLK(slot) do { } while (0)
+#define MIP_STAMP(slot) do { } while (0)
+#endif
+
 struct TileCoord {
     int m0, n0, kb_begin, kb_end;
 };
@@ -90,6 +99,108 @@ __device__ __forceinline__ void store_chunk(const DenseParams& p, int32_t* dst, 
     }
 }
 
+// Adds one 32 x 32 chunk (thread = row, v = its 32 columns) into C through the TMA: the rows
+// go to a 128-byte-swizzled staging buffer, then one elected lane issues a tile reduce-add
+// (32-bit integer adds performed at the L2: exact and order-independent), which clips the
+// tile at the edges of C.  Used for split-K.  `buf` alternates between two buffers; at most
+// one earlier copy may still be reading shared memory.
+__device__ __forceinline__ void tma_reduce_chunk(const DenseParams& p, uint32_t buf, const uint32_t (&v)[32],
+                                                 int lane, int x, int y) {
+    if (elect_one()) tma_store_wait_read<1>();
+    __syncwarp();
+    const uint32_t row = buf + static_cast<uint32_t>(lane) * 128u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) st_shared_v4(row + (static_cast<uint32_t>(j ^ (lane & 7)) << 4), &v[4 * j]);
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (elect_one()) {   // always the same lane: bulk-group bookkeeping is per thread
+        tma_reduce_add_2d(&p.tmap_c, buf, x, y);
+        tma_store_commit();
+    }
+}
+
+// Stores one 128 x 32 slab of the tile (all four epilogue warps, thread = row) with a single
+// TMA tile store: the rows go to a 128-byte-swizzled 16 KB staging buffer, the four warps
+// meet at a named barrier, and one thread issues the store, which clips at the edges of C.
+// `buf` alternates between two buffers; `issuer` is true in exactly one warp.
+__device__ __forceinline__ void tma_store_slab(const DenseParams& p, uint32_t buf, const uint32_t (&v)[32],
+                                               int lane, int q, bool issuer, int x, int y) {
+    if (issuer && elect_one()) tma_store_wait_read<1>();
+    asm volatile("bar.sync 1, 128;" ::: "memory");      // the buffer is free for all four warps
+    const int r = q * 32 + lane;
+    const uint32_t row = buf + static_cast<uint32_t>(r) * 128u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) st_shared_v4(row + (static_cast<uint32_t>(j ^ (r & 7)) << 4), &v[4 * j]);
+    fence_proxy_async_smem();
+    asm volatile("bar.sync 1, 128;" ::: "memory");      // all 128 rows are in place
+    if (issuer && elect_one()) {
+        tma_store_2d(&p.tmap_c, buf, x, y);
+        tma_store_commit();
+    }
+}
+
+// Writes one 32 x 32 chunk (thread = row, v = its 32 columns) with fully coalesced 16-byte
+// accesses: the chunk is transposed through a swizzled staging buffer so that every store
+// instruction of the warp covers four complete 128-byte rows of C.  With accumulate, the
+// incoming C is read with the same access pattern and added.  Needs a 16-byte aligned C
+// base and ldc % 4 == 0.  (row0, col0) is the chunk's origin in C.
+__device__ __forceinline__ void coalesced_chunk(const DenseParams& p, uint32_t buf, const uint32_t (&v)[32],
+                                                int lane, int row0, int col0) {
+    MIP_CLK(24);
+    __syncwarp();   // the previous chunk's reads of `buf` are done
+    MIP_CLK(25);
+    const uint32_t mine = buf + static_cast<uint32_t>(lane) * 128u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) st_shared_v4(mine + (static_cast<uint32_t>(j ^ (lane & 7)) << 4), &v[4 * j]);
+    MIP_CLK(26);
+    __syncwarp();
+    MIP_CLK(27);
+    const int piece = lane & 7;                 // which 16 bytes (4 columns) of a row
+    const int col = col0 + 4 * piece;
+    const int cols_left = p.N - col;            // <= 0: nothing of this piece is inside C
+    // all eight shared-memory reads are issued before the first global access depends on them
+    uint32_t x[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = 4 * i + (lane >> 3);
+        asm("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+            : "=r"(x[i][0]), "=r"(x[i][1]), "=r"(x[i][2]), "=r"(x[i][3])
+            : "r"(buf + static_cast<uint32_t>(r) * 128u + (static_cast<uint32_t>(piece ^ (r & 7)) << 4))
+            : "memory");
+    }
+    int32_t* dst0 = p.C + static_cast<long long>(row0 + (lane >> 3)) * p.ldc + col;
+    const long long step = 4 * p.ldc;
+    if (p.accumulate && cols_left >= 4) {
+        uint32_t c[8][4];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (row0 + 4 * i + (lane >> 3) < p.M) ld_global_v4(dst0 + i * step, c[i]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) x[i][j] += c[i][j];
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int row = row0 + 4 * i + (lane >> 3);
+        if (row < p.M && cols_left > 0) {
+            int32_t* dst = dst0 + i * step;
+            if (cols_left >= 4) {
+                st_global_v4(dst, x[i]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 3; ++j) {
+                    if (j < cols_left) {
+                        uint32_t y = x[i][j];
+                        if (p.accumulate) y += static_cast<uint32_t>(dst[j]);
+                        dst[j] = static_cast<int32_t>(y);
+                    }
+                }
+            }
+        }
+    }
+}
+
 template <bool kPair>
 __global__ void __launch_bounds__(kDenseThreads, 1)
 mip_dense_kernel(const __grid_constant__ DenseParams p) {
@@ -100,6 +211,10 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
     const int first_unit = kPair ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
     const int unit_stride = kPair ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
     const int b_rows = kPair ? (p.block_n >> 1) : p.block_n;   // rows of B staged by this CTA
+    MIP_STAMP(0);
+#ifdef MIPGEMM_TRACE
+    if (threadIdx.x < 32) mip_trace_smem[threadIdx.x] = 0;
+#endif
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
@@ -109,14 +224,16 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
     const uint32_t a_bytes = kBlockM * p.block_k;
     const uint32_t b_bytes = b_rows * p.block_k;
     const uint32_t stage_bytes = a_bytes + b_bytes;
-    const uint32_t ctrl = smem_base + p.stages * stage_bytes;
+    // shared memory: [stages x (A tile | B tile)] [epilogue staging] [control block]
+    const uint32_t staging = smem_base + p.stages * stage_bytes;
+    const uint32_t ctrl = staging + kStagingBytes;
     // control block: full[stages] | empty[stages] | tmem_full[2] | tmem_empty[2] | drain | slot | abort
     const uint32_t bar_full = ctrl;
     const uint32_t bar_empty = bar_full + 8u * p.stages;
     const uint32_t bar_tfull = bar_empty + 8u * p.stages;
     const uint32_t bar_tempty = bar_tfull + 16u;
     const uint32_t bar_drain = bar_tempty + 16u;
-    uint8_t* ctrl_ptr = smem + p.stages * stage_bytes;
+    uint8_t* ctrl_ptr = smem + p.stages * stage_bytes + kStagingBytes;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl_ptr + 16 * p.stages + 40);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
 
@@ -140,6 +257,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         fence_mbar_init();
         tma_prefetch_desc(&p.tmap_a);
         tma_prefetch_desc(&p.tmap_b);
+        if (p.c_mode == 1 || p.c_mode == 2) tma_prefetch_desc(&p.tmap_c);
     }
     if (warp == 1) {
         tmem_alloc<kGroup>(smem_u32(tmem_slot), p.tmem_cols);
@@ -153,6 +271,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
     }
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) MIP_STAMP(1);
 
     const int total_units = p.tiles_m * p.tiles_n * p.split_k;
     const uint64_t budget = p.wait_budget_ns;
@@ -212,6 +331,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     else
                         tma_load_2d(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta);
                 }
+                if (issued == 0) MIP_STAMP(2);
                 if (p.a_im2col && ++cc == p.c_chunks) {   // next filter tap (r, s)
                     cc = 0;
                     if (++fs == p.conv_s) { fs = 0; ++fr; }
@@ -250,6 +370,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 const uint32_t d_tmem = tmem_base + acc * p.block_n;
                 for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb) {
                     if (!mbar_wait(bar_full + 8u * s, phase, abort_flag, budget)) { ok = false; break; }
+                    if (t == 0 && kb == tc.kb_begin) MIP_STAMP(3);
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * stage_bytes;
                     const uint64_t a_desc = make_kmajor_desc(a_addr, p.block_k);
@@ -270,6 +391,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     }
                     if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
                 }
+                if (t == 0) MIP_STAMP(4);
                 if (ok) {
                     const uint32_t tfull_local = bar_tfull + 8u * acc;
                     const uint32_t tfull_peer = kPair ? mapa_u32(tfull_local, 1) : 0u;
@@ -302,21 +424,45 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
             const uint32_t acc = t & 1, acc_phase = (t >> 1) & 1;
             if (!mbar_wait(bar_tfull + 8u * acc, acc_phase, abort_flag, budget)) break;
+            if (t == 0 && warp == 2) MIP_STAMP(5);
+            MIP_CLK(20);
             tc_fence_after();
             const int m_cta = tc.m0 + static_cast<int>(cta_rank) * kBlockM;
             const int row = m_cta + q * 32 + lane;
             const int n_rem = p.N - tc.n0;
             const int n_here = min(p.block_n, n_rem);
-            if (m_cta + q * 32 < p.M) {
+            if (p.c_mode == 1 || m_cta + q * 32 < p.M) {   // (slab stores need all four warps)
                 int32_t* crow = p.C + static_cast<long long>(row) * p.ldc + tc.n0;
                 const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.block_n;
-                for (int c0 = 0; c0 < n_here; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld_32x32(t_row + c0, v);
+                const uint32_t my_staging = staging + static_cast<uint32_t>(q) * 8192u;
+                // two register buffers: the TMEM load of the next chunk is in flight while the
+                // current one is written out
+                uint32_t va[32], vb[32];
+                MIP_CLK(21);
+                tmem_ld_32x32(t_row, va);
+                MIP_CLK(22);
+                for (int c0 = 0; c0 < n_here; c0 += 64) {
                     tmem_ld_wait();
-                    if (row < p.M) store_chunk(p, crow + c0, v, min(32, n_here - c0));
+                    MIP_CLK(23);
+                    if (c0 + 32 < n_here) tmem_ld_32x32(t_row + c0 + 32, vb);
+                    if (p.c_mode == 1) tma_store_slab(p, staging, va, lane, q, warp == 2, tc.n0 + c0, m_cta);
+                    else if (p.c_mode == 3) coalesced_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0);
+                    else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging, va, lane, tc.n0 + c0, m_cta + q * 32);
+                    else if (row < p.M) store_chunk(p, crow + c0, va, min(32, n_here - c0));
+                    MIP_CLK(28);
+                    if (c0 + 32 < n_here) {
+                        tmem_ld_wait();
+                        MIP_CLK(29);
+                        if (c0 + 64 < n_here) tmem_ld_32x32(t_row + c0 + 64, va);
+                        if (p.c_mode == 1) tma_store_slab(p, staging + 16384u, vb, lane, q, warp == 2, tc.n0 + c0 + 32, m_cta);
+                        else if (p.c_mode == 3) coalesced_chunk(p, my_staging + 4096u, vb, lane, m_cta + q * 32, tc.n0 + c0 + 32);
+                        else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + 4096u, vb, lane, tc.n0 + c0 + 32, m_cta + q * 32);
+                        else if (row < p.M) store_chunk(p, crow + c0 + 32, vb, min(32, n_here - c0 - 32));
+                    }
                 }
             }
+            MIP_CLK(30);
+            if (warp == 2) { if (t == 0) MIP_STAMP(6); MIP_STAMP(7); }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
@@ -324,10 +470,13 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 else mbar_arrive(bar_tempty + 8u * acc);
             }
         }
+        // every tile copy issued by this warp must be complete before the CTA may exit
+        if ((p.c_mode == 2 || (p.c_mode == 1 && warp == 2)) && elect_one()) tma_store_wait<0>();
     }
 
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) MIP_STAMP(8);
     if (kPair) {   // neither CTA may leave while the other can still reach its shared memory
         cluster_arrive();
         cluster_wait();
@@ -336,6 +485,10 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         tc_fence_after();
         tmem_dealloc<kGroup>(tmem_base, p.tmem_cols);
     }
+    if (threadIdx.x == 0) MIP_STAMP(9);
+#ifdef MIPGEMM_TRACE
+    if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) for (int i = 20; i < 32; ++i) p.trace[i] = mip_trace_smem[i];
+#endif
     if (threadIdx.x == 0 && *abort_flag != 0) atomicOr(p.status, 1u);
 }
 

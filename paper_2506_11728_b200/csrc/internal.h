@@ -11,12 +11,18 @@ constexpr int kBlockM = 128;          // rows of C per CTA (TMEM lanes)
 constexpr int kDenseThreads = 192;    // producer warp, MMA warp, 4 epilogue warps
 constexpr int kMaxStages = 12;
 constexpr int kCtrlBytes = 512;       // barriers + TMEM slot + abort word
+constexpr int kStagingBytes = 4 * 2 * 4096;   // epilogue: 4 warps x 2 buffers x (32 rows x 128 B)
+#ifdef MIPGEMM_TRACE
+constexpr int kSmemBudget = 226 * 1024;   // leaves room for the static trace array
+#else
 constexpr int kSmemBudget = 227 * 1024;
+#endif
 
 // Everything the dense kernel needs; passed by value as a __grid_constant__.
 struct alignas(64) DenseParams {
     CUtensorMap tmap_a;      // tiled {K, M} byte tensor, or im2col-mode NHWC tensor
     CUtensorMap tmap_b;      // tiled {K, N} byte tensor (weights, K contiguous)
+    CUtensorMap tmap_c;      // tiled {N, M} int32 tensor, 32 x 32 boxes (used when c_mode == 2)
     int32_t* C;
     long long ldc;
     int M, N;
@@ -30,6 +36,9 @@ struct alignas(64) DenseParams {
     int accumulate;          // epilogue adds the incoming C
     int use_red;             // epilogue reduces with red.global.add (split-K)
     int store_vec;           // 8, 4 or 1 int32 per store instruction
+    int c_mode;              // 0: row-per-thread stores (any alignment), 1: coalesced stores through
+                             // shared memory, 2: TMA tile reduce-add (split-K); 1 and 2 need a 16-byte
+                             // aligned C base and ldc % 4 == 0
     uint32_t idesc;          // tcgen05 instruction descriptor
     uint32_t tmem_cols;      // power of two >= 2*block_n
     // implicit im2col (operand A gathered by TMA im2col loads)
@@ -38,6 +47,7 @@ struct alignas(64) DenseParams {
     int stride_w, stride_h, pad_w, pad_h, dil_w, dil_h;
     unsigned int* status;    // device word, bit 0 set when a bounded wait expired
     unsigned long long wait_budget_ns;
+    unsigned long long* trace;   // timeline stamps of CTA 0; only read by builds with -DMIPGEMM_TRACE
 };
 
 cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream);

@@ -109,3 +109,15 @@ def test_resnet50_layers_batch32_sampled_images(mg, layer):
     for n in (0, 17, Nb - 1):
         want = orc.conv(X[n:n + 1], Wt, stride=(st, st), pad=(pd, pd))
         assert np.array_equal(got[n:n + 1], want), "image %d: %s" % (n, first_mismatch(got[n:n + 1], want))
+
+
+@pytest.mark.parametrize("case", TMA_CASES[:4] + TMA_CASES[6:7])
+def test_implicit_im2col_cta_pair(mg, case):
+    Nb, H, W, Cin, Cout, R, S, stride, pad, dil = case
+    mg.mipgemm_set_tuning(force_path=mg.PATH_DENSE_PAIR)
+    try:
+        p = check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=40, expect_flag=mg.PATH_IM2COL_TMA)
+        assert p & mg.PATH_MASK == mg.PATH_DENSE_PAIR
+        check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=41, accumulate=True)
+    finally:
+        mg.mipgemm_set_tuning()

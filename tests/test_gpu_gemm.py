@@ -221,3 +221,29 @@ def test_lent_workspace(mg):
         assert mg.mipgemm_u8s8s32(130, 70, 100, dA, 101, dB, 103, dC, 71, 0, check=False) == mg.ERR_WORKSPACE
     finally:
         mg.mipgemm_set_workspace(None, 0)
+
+
+@pytest.mark.parametrize("mode", ["s8", "u8"])
+@pytest.mark.parametrize("accumulate", [False, True])
+def test_ragged_shapes_cta_pair_kernel(mg, mode, accumulate):
+    """The cta_group::2 form on shapes that leave the second CTA of a pair partly or wholly empty."""
+    mg.mipgemm_set_tuning(force_path=mg.PATH_DENSE_PAIR)
+    try:
+        for i, (M, N, K) in enumerate(RAGGED + [(513, 300, 272), (1000, 3000, 784)]):
+            check_case(mg, mode, M, N, K, accumulate=accumulate, seed=400 + i, expect_path=mg.PATH_DENSE_PAIR)
+        for bn in (64, 128):
+            mg.mipgemm_set_tuning(block_n=bn, force_path=mg.PATH_DENSE_PAIR)
+            check_case(mg, mode, 700, 600, 1424, accumulate=accumulate, seed=450 + bn, ldc=604,
+                       expect_path=mg.PATH_DENSE_PAIR)
+    finally:
+        mg.mipgemm_set_tuning()
+
+
+def test_cta_pair_with_unaligned_c_and_repack(mg):
+    mg.mipgemm_set_tuning(force_path=mg.PATH_DENSE_PAIR)
+    try:
+        path = check_case(mg, "s8", 1000, 3001, 777, lda=777, ldb=777, ldc=3001, accumulate=True, seed=460)
+        assert path & mg.PATH_REPACK and path & mg.PATH_MASK == mg.PATH_DENSE_PAIR
+        check_case(mg, "u8", 515, 259, 400, ldc=261, seed=461)
+    finally:
+        mg.mipgemm_set_tuning()
