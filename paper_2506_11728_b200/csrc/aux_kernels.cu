@@ -118,14 +118,108 @@ __global__ void mip_im2col_kernel(const Im2colParams p, long long chunks_per_row
     }
 }
 
+// Row-staged variant for channel counts TMA cannot address (e.g. the 3-channel stem): one CTA
+// per output row (n, ho).  The R input rows that the row needs are staged in shared memory
+// between zero margins as wide as the padding (rows outside the image are all zeros), so no
+// bounds check is left in the inner loop.  Thread t serves 16-byte chunk t % chunks of the
+// augmented-matrix row of every (t / chunks)-th pixel: the 16 source offsets of its chunk
+// are computed once and kept in registers, and the chunks leave with coalesced 16-byte stores.
+__global__ void __launch_bounds__(256)
+mip_im2col_rows_kernel(const Im2colParams p, int row_pitch, int margin, int left_pad, int stage_vec,
+                       int ho_per_cta, int staged_rows) {
+    extern __shared__ __align__(16) uint8_t rows[];                      // [staged_rows][row_pitch]
+    const int groups = static_cast<int>((p.Ho + ho_per_cta - 1) / ho_per_cta);
+    const long long n = blockIdx.x / groups;
+    const int ho0 = static_cast<int>(blockIdx.x - n * groups) * ho_per_cta;
+    const int Cin = static_cast<int>(p.Cin), Wo = static_cast<int>(p.Wo);
+    const int K = static_cast<int>(p.k_real), chunks = static_cast<int>(p.k_pitch / 16);
+    const int data_bytes = static_cast<int>(p.W) * Cin;
+
+    for (int i = threadIdx.x; i < staged_rows * row_pitch / 16; i += blockDim.x)
+        reinterpret_cast<uint4*>(rows)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    // staged row q holds input row h0 + q, h0 = first row the CTA's first output row touches
+    const long long h0 = static_cast<long long>(ho0) * p.stride_h - p.pad_h;
+    for (int q = 0; q < staged_rows; ++q) {
+        const long long h = h0 + q;
+        if (h < 0 || h >= p.H) continue;
+        const uint8_t* src = p.X + ((n * p.H + h) * p.W) * p.Cin;
+        uint8_t* dst = rows + q * row_pitch + margin;      // 16-byte aligned
+        if (stage_vec) {
+            for (int i = threadIdx.x; i < data_bytes / 16; i += blockDim.x)
+                reinterpret_cast<uint4*>(dst)[i] = __ldg(reinterpret_cast<const uint4*>(src) + i);
+        } else {
+            for (int i = threadIdx.x; i < data_bytes; i += blockDim.x) dst[i] = __ldg(src + i);
+        }
+    }
+
+    const int j = threadIdx.x % chunks;                // this thread's chunk of every pixel row
+    const int lane_px = threadIdx.x / chunks;
+    const int px_step = blockDim.x / chunks;
+    int off[16];
+#pragma unroll
+    for (int b = 0; b < 16; ++b) {
+        const int k = j * 16 + b;
+        if (k < K) {
+            const int tap = k / Cin, c = k - tap * Cin;
+            const int r = tap / p.S, s = tap - r * p.S;
+            off[b] = r * p.dil_h * row_pitch + s * p.dil_w * Cin + c;   // relative to the window start
+        } else {
+            off[b] = -1;
+        }
+    }
+    __syncthreads();
+
+    const int ho_end = min(ho0 + ho_per_cta, static_cast<int>(p.Ho));
+    if (lane_px < px_step) {
+        for (int ho = ho0; ho < ho_end; ++ho) {
+            uint8_t* out_row = p.out + ((n * p.Ho + ho) * p.Wo) * p.k_pitch;
+            const int row_base = (ho - ho0) * p.stride_h * row_pitch + margin - left_pad;
+            for (int wo = lane_px; wo < Wo; wo += px_step) {
+                const int base = row_base + wo * p.stride_w * Cin;      // window start in the staged rows
+                uint32_t words[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (int b = 0; b < 16; ++b)
+                    if (off[b] >= 0) words[b >> 2] |= static_cast<uint32_t>(rows[base + off[b]]) << (8 * (b & 3));
+                *reinterpret_cast<uint4*>(out_row + (static_cast<long long>(wo) * chunks + j) * 16) =
+                    make_uint4(words[0], words[1], words[2], words[3]);
+            }
+        }
+    }
+}
+
 cudaError_t launch_im2col(const Im2colParams& p, cudaStream_t stream) {
     const long long M = p.Nb * p.Ho * p.Wo;
     if (M <= 0) return cudaSuccess;
+    const bool vec = (p.Cin % 16 == 0) && (reinterpret_cast<uintptr_t>(p.X) % 16 == 0);
+    // padded row: [margin >= pad_w*Cin zeros, 16-byte multiple][W*Cin bytes][zeros up to the last
+    // window's end]
+    const long long left_pad = static_cast<long long>(p.pad_w) * p.Cin;
+    const long long margin = (left_pad + 15) & ~15LL;
+    const long long last_end = margin - left_pad +
+                               ((p.Wo - 1) * p.stride_w + static_cast<long long>(p.S - 1) * p.dil_w + 1) * p.Cin;
+    const long long need = margin + p.W * p.Cin > last_end ? margin + p.W * p.Cin : last_end;
+    const long long row_pitch = (need + 15) & ~15LL;
+    const int stage_vec = ((p.W * p.Cin) % 16 == 0 && reinterpret_cast<uintptr_t>(p.X) % 16 == 0) ? 1 : 0;
+    // several output rows per CTA share their staged input rows and the per-thread set-up
+    int ho_per_cta = 4;
+    long long staged = (ho_per_cta - 1LL) * p.stride_h + (p.R - 1LL) * p.dil_h + 1;
+    while (ho_per_cta > 1 && staged * row_pitch > 48 * 1024) {
+        --ho_per_cta;
+        staged = (ho_per_cta - 1LL) * p.stride_h + (p.R - 1LL) * p.dil_h + 1;
+    }
+    const long long smem = staged * row_pitch;
+    const long long grid = p.Nb * ((p.Ho + ho_per_cta - 1) / ho_per_cta);
+    if (!vec && smem <= 48 * 1024 && grid < 0x7FFFFFFFLL && p.k_pitch / 16 <= 256) {
+        mip_im2col_rows_kernel<<<static_cast<unsigned>(grid), 256, static_cast<size_t>(smem), stream>>>(
+            p, static_cast<int>(row_pitch), static_cast<int>(margin), static_cast<int>(left_pad), stage_vec,
+            ho_per_cta, static_cast<int>(staged));
+        return cudaGetLastError();
+    }
     const long long chunks = p.k_pitch / 16;
     const long long total = M * chunks;
     const int threads = 256;
     const long long blocks = min((total + threads - 1) / threads, 148LL * 32);
-    const bool vec = (p.Cin % 16 == 0) && (reinterpret_cast<uintptr_t>(p.X) % 16 == 0);
     if (vec)
         mip_im2col_kernel<true><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(p, chunks, total);
     else
