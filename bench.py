@@ -35,7 +35,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM traffic (bytes read + written) of the dominant kernel per launch, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that workload).
-NCU_TRAFFIC_BYTES = {"square": None, "bert": None, "resnet": None, "skinny": None}
+NCU_TRAFFIC_BYTES = {
+    "square": 1561e6,   # profiles/dense_kernel_square_sweep.md: (6.4 + 8.4 + 55.3 + 606.3 + 7128.4) MB / 5 launches
+    "bert": None,
+    "resnet": None,
+    "skinny": 58.9e6,   # profiles/skinny_kernel_14336x4096.md: one 14336 x 4096 launch (traffic = algorithmic bytes)
+}
 
 
 def load_peaks():
@@ -312,6 +317,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--detail", action="store_true", help="print per-problem timings to stderr")
     ap.add_argument("--eager", action="store_true", help="plain launches instead of CUDA-graph replay")
+    ap.add_argument("--only", default="", help="keep only problems whose name contains this text (for profiling)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -354,6 +360,12 @@ def main():
         workload = "skinny decode GEMMs s8*s8->s32, M in %s, weights %s, rotated over >=512 MB" % (
             inputs.SKINNY_M, inputs.SKINNY_WEIGHTS)
         unit, metric = "GB/s", "skinny_gemm_gbs"
+
+    if args.only:
+        probs = [p for p in probs if args.only in p.name]
+        workload += " [only: %s]" % args.only
+        if not probs:
+            raise SystemExit("--only matched no problem")
 
     # launch order of one step: every problem once (resnet: layer multiplicity; skinny: all
     # rotation slots), grouped per problem so one event pair brackets each group
