@@ -63,7 +63,9 @@ typedef enum {
     MIPGEMM_ERR_UNSUPPORTED = 3, /* current device is not compute capability 10.0                  */
     MIPGEMM_ERR_WORKSPACE = 4,   /* scratch memory could not be obtained / lent buffer too small   */
     MIPGEMM_ERR_CUDA = 5,        /* a CUDA call failed; see mipgemm_last_cuda_error()              */
-    MIPGEMM_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (kernel returned early)     */
+    MIPGEMM_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (kernel returned early)     */
+    MIPGEMM_ERR_STATIC_SCRATCH_LIMIT = 7 /* mipgemm_s8s8s32_static_scratch: operands too large for  */
+                                         /* the built-in scratch array (nothing was enqueued)        */
 } mipgemm_status_t;
 
 /* Which kernel family served the most recent GEMM/conv call of this thread (test hook). */
@@ -139,6 +141,46 @@ int mipgemm_host_s8s8s32(int64_t M, int64_t N, int64_t K,
 int mipgemm_host_u8s8s32(int64_t M, int64_t N, int64_t K,
                          const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
                          int32_t *C, int64_t ldc, int accumulate, void *stream);
+
+/*
+ * Allocation-free variant of mipgemm_s8s8s32 (the paper has no counterpart: this is an
+ * integration aid, not part of the method).
+ *
+ * Who needs it: callers that are not allowed to reach the CUDA allocator -- code embedded
+ * in a memory-planned inference runtime that owns the whole device, real-time loops that
+ * must never block in cudaMalloc/cudaFree, plug-ins running under another framework's
+ * memory pool.  The other entry points take scratch memory with cudaMallocAsync whenever
+ * an operand has to be re-pitched for the tensor-memory-accelerator (base or pitch not a
+ * multiple of 16 bytes) and allocate one status word per device on first use; this one
+ * calls no allocating routine at all.  Its re-pitching scratch is a fixed array of
+ * MIPGEMM_STATIC_SCRATCH_BYTES that lives in the library image: every GPU that loads
+ * libmipgemm holds that much memory until the process exits, used or not.
+ *
+ * Same arguments, layouts, exactness contract and return codes as mipgemm_s8s8s32 (all
+ * pointers are device pointers; C is read only when accumulate != 0), with these
+ * differences:
+ *  - It always runs the dense tensor-core kernel (no skinny-M shortcut).
+ *  - If the operands that need re-pitching take more than MIPGEMM_STATIC_SCRATCH_BYTES
+ *    (A needs M*roundup(K,16) bytes when A or lda is not 16-byte aligned, B needs
+ *    N*roundup(K,16) likewise, each rounded up to 256) the call returns
+ *    MIPGEMM_ERR_STATIC_SCRATCH_LIMIT and enqueues nothing.
+ *  - The first call on each device performs a one-time set-up (it looks up the device
+ *    address of the array and sets kernel attributes).  Make that first call outside any
+ *    stream capture.
+ *  - All calls on a device share the one array.  It keeps whatever the previous call left
+ *    in it; that is harmless because each call overwrites every byte it later reads, so
+ *    nothing has to be cleared between calls.  But two calls whose kernels can overlap on
+ *    the GPU (different streams, or several host threads) race on the array and corrupt
+ *    each other's operands: order such calls on one stream or serialise them yourself.
+ *  - A bounded device-side wait that expires in this path sets a word private to this
+ *    entry point; mipgemm_device_status() does not report it.
+ */
+#define MIPGEMM_STATIC_SCRATCH_BYTES (8u << 20)
+int mipgemm_s8s8s32_static_scratch(int64_t M, int64_t N, int64_t K,
+                                   const int8_t *A, int64_t lda,
+                                   const int8_t *B, int64_t ldb,
+                                   int32_t *C, int64_t ldc,
+                                   int accumulate, void *stream);
 
 /* ---- support calls (no counterpart in the paper) ---- */
 

@@ -24,6 +24,8 @@ _lib = ctypes.CDLL(LIB_PATH)
 _i64, _int, _vp, _sz = ctypes.c_int64, ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t
 
 OK, ERR_INVALID_ARG, ERR_K_TOO_LARGE, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
+ERR_STATIC_SCRATCH_LIMIT = 7
+STATIC_SCRATCH_BYTES = 8 << 20
 PATH_NONE, PATH_DENSE, PATH_DENSE_PAIR, PATH_SKINNY, PATH_TRIVIAL = range(5)
 PATH_MASK = 0xFF
 PATH_REPACK, PATH_SPLITK, PATH_IM2COL_TMA, PATH_IM2COL_EXPLICIT = 0x100, 0x200, 0x400, 0x800
@@ -35,6 +37,7 @@ SIGNATURES = {
     "mipgemm_conv_u8s8s32": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, _int, _vp]),
     "mipgemm_host_s8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_host_u8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
+    "mipgemm_s8s8s32_static_scratch": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_launch_count": (ctypes.c_uint64, []),
     "mipgemm_device_status": (_int, [_vp]),
     "mipgemm_set_workspace": (_int, [_vp, _sz]),
@@ -113,6 +116,16 @@ def mipgemm_host_s8s8s32(M, N, K, A, lda, B, ldb, C, ldc, accumulate=0, stream=N
 def mipgemm_host_u8s8s32(M, N, K, A, lda, B, ldb, C, ldc, accumulate=0, stream=None, check=True) -> int:
     return _check(_lib.mipgemm_host_u8s8s32(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
                                             int(bool(accumulate)), _stream(stream)), check)
+
+
+def mipgemm_s8s8s32_static_scratch(M, N, K, A, lda, B, ldb, C, ldc, accumulate=0, stream=None, check=True) -> int:
+    """mipgemm_s8s8s32 for callers that may not allocate device memory: re-pitching scratch comes from
+    a fixed STATIC_SCRATCH_BYTES array inside the library (one per GPU, shared by all calls -- calls
+    that can overlap on the GPU race on it).  Returns ERR_STATIC_SCRATCH_LIMIT, having launched
+    nothing, when the operands need more than that.  Make the first call on a device outside any
+    stream capture."""
+    return _check(_lib.mipgemm_s8s8s32_static_scratch(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                                      int(bool(accumulate)), _stream(stream)), check)
 
 
 def mipgemm_launch_count() -> int:

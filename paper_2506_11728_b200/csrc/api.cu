@@ -660,6 +660,8 @@ const char* mipgemm_status_string(int status) {
         case MIPGEMM_ERR_WORKSPACE: return "scratch memory unavailable or lent buffer too small";
         case MIPGEMM_ERR_CUDA: return "CUDA call failed";
         case MIPGEMM_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case MIPGEMM_ERR_STATIC_SCRATCH_LIMIT:
+            return "operands need more re-pitching scratch than the built-in static buffer holds";
         default: return "unknown status";
     }
 }
@@ -691,3 +693,144 @@ int mipgemm_set_tuning(int block_n, int stages, int split_k, int force_path) {
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free GEMM entry point.
+//
+// Everything above obtains its scratch memory (and one status word per device) from the
+// CUDA allocator.  Some callers cannot do that: code running inside a memory-planned
+// inference runtime that owns every byte of the device, a real-time loop that must never
+// enter the driver's allocator, a process whose memory pool has been handed over entirely
+// to another framework.  For them the re-pitching GEMM exists once more below with its
+// scratch in a fixed array that is part of the library image on every GPU that loads it.
+// Nothing on this path calls cudaMalloc, cudaMallocAsync, cudaFree or any other allocating
+// routine; it shares no state with the entry points above.
+// ---------------------------------------------------------------------------------------
+namespace {
+
+// The scratch itself.  Host code must never use this name as an address: on the host it is
+// only a handle for cudaGetSymbolAddress (see noalloc_device()).
+static __device__ __align__(256) unsigned char g_static_scratch[MIPGEMM_STATIC_SCRATCH_BYTES];
+// Word that receives the "bounded wait expired" flag of kernels launched from this path.
+static __device__ unsigned int g_static_status;
+
+struct NoAllocDevice {
+    bool ready = false;
+    int status = MIPGEMM_OK;
+    DeviceState st;                 // sm_count, pair_clusters, status_word (-> g_static_status)
+    unsigned char* scratch = nullptr;   // device address of g_static_scratch on this device
+};
+NoAllocDevice g_noalloc[kMaxDevices];
+std::mutex g_noalloc_mutex;
+
+// Per-device set-up, done by the first call on each device with that device current:
+// capability check, tensor-map encoders, kernel attributes and the DEVICE addresses of the
+// two static symbols.  No allocation.
+int noalloc_device(NoAllocDevice** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return MIPGEMM_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    NoAllocDevice& d = g_noalloc[dev];
+    if (!d.ready) {
+        int major = 0, minor = 0;
+        if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&d.st.sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return cuda_fail(e);
+        if (major != 10 || minor != 0) {
+            d.status = MIPGEMM_ERR_UNSUPPORTED;
+        } else {
+            {
+                std::lock_guard<std::mutex> lock2(g_mutex);   // the encoder pointers are shared
+                if (!g_encode_tiled) {
+                    void* fn = nullptr;
+                    cudaDriverEntryPointQueryResult qr;
+                    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr);
+                    if (e != cudaSuccess || qr != cudaDriverEntryPointSuccess || !fn)
+                        return cuda_fail(e == cudaSuccess ? cudaErrorUnknown : e);
+                    g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+                }
+            }
+            if ((e = dense_init()) != cudaSuccess) return cuda_fail(e);
+            d.st.pair_clusters = dense_pair_max_clusters(kSmemBudget);
+            void* ptr = nullptr;
+            if ((e = cudaGetSymbolAddress(&ptr, g_static_scratch)) != cudaSuccess) return cuda_fail(e);
+            d.scratch = static_cast<unsigned char*>(ptr);
+            ptr = nullptr;
+            if ((e = cudaGetSymbolAddress(&ptr, g_static_status)) != cudaSuccess) return cuda_fail(e);
+            d.st.status_word = static_cast<unsigned int*>(ptr);
+            d.status = MIPGEMM_OK;
+        }
+        d.ready = true;
+    }
+    *out = &d;
+    return d.status;
+}
+
+}  // namespace
+
+extern "C" int mipgemm_s8s8s32_static_scratch(int64_t M, int64_t N, int64_t K, const int8_t* A, int64_t lda,
+                                              const int8_t* B, int64_t ldb, int32_t* C, int64_t ldc,
+                                              int accumulate, void* stream_v) {
+    if (M < 0 || N < 0 || K < 0) return MIPGEMM_ERR_INVALID_ARG;
+    if (M > 0x7FFFFF00LL || N > 0x7FFFFF00LL) return MIPGEMM_ERR_INVALID_ARG;
+    if (lda < K || ldb < K || ldc < N) return MIPGEMM_ERR_INVALID_ARG;
+    if (K > 131071) return MIPGEMM_ERR_K_TOO_LARGE;
+    if (M == 0 || N == 0) return MIPGEMM_OK;
+    if (!C || reinterpret_cast<uintptr_t>(C) % 4 != 0) return MIPGEMM_ERR_INVALID_ARG;
+    if (K > 0 && (!A || !B)) return MIPGEMM_ERR_INVALID_ARG;
+    // How much of the static array this call needs; refuse before anything is enqueued.
+    const size_t need = gemm_scratch_bytes(M, N, K, A, lda, B, ldb);
+    if (need > static_cast<size_t>(MIPGEMM_STATIC_SCRATCH_BYTES)) return MIPGEMM_ERR_STATIC_SCRATCH_LIMIT;
+
+    NoAllocDevice* nd = nullptr;
+    int st = noalloc_device(&nd);
+    if (st != MIPGEMM_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    cudaError_t e;
+    if (K == 0) {
+        if (!accumulate) {
+            if ((e = launch_fill_zero(C, ldc, M, N, stream)) != cudaSuccess) return cuda_fail(e);
+            ++g_launches;
+        }
+        return MIPGEMM_OK;
+    }
+
+    // Re-pitch whatever TMA cannot address into the static array.  Every byte the GEMM kernel
+    // will read from the array (K bytes of M, respectively N, rows) is written here first, so
+    // nothing left behind by an earlier call can reach the result and nothing needs clearing.
+    const long long pitch = round_up(K, 16);
+    const void* a_use = A;
+    const void* b_use = B;
+    long long lda_use = lda, ldb_use = ldb;
+    size_t used = 0;
+    if (!aligned16(A, lda)) {
+        unsigned char* dst = nd->scratch + used;
+        used += align256(static_cast<size_t>(M) * pitch);
+        if ((e = launch_repack(A, lda, dst, pitch, M, K, stream)) != cudaSuccess) return cuda_fail(e);
+        ++g_launches;
+        a_use = dst;
+        lda_use = pitch;
+    }
+    if (!aligned16(B, ldb)) {
+        unsigned char* dst = nd->scratch + used;
+        used += align256(static_cast<size_t>(N) * pitch);
+        if ((e = launch_repack(B, ldb, dst, pitch, N, K, stream)) != cudaSuccess) return cuda_fail(e);
+        ++g_launches;
+        b_use = dst;
+        ldb_use = pitch;
+    }
+
+    const int block_k = 128;
+    const Plan pl = make_plan(M, N, K, block_k, &nd->st);
+    DenseParams p;
+    std::memset(&p, 0, sizeof(p));
+    fill_common(p, pl, M, N, C, ldc, block_k, false, accumulate, &nd->st);
+    if ((st = encode_tiled_2d(&p.tmap_a, a_use, K, M, lda_use, block_k, kBlockM)) != MIPGEMM_OK) return st;
+    if ((st = encode_tiled_2d(&p.tmap_b, b_use, K, N, ldb_use, block_k, pl.pair ? pl.block_n / 2 : pl.block_n)) !=
+        MIPGEMM_OK)
+        return st;
+    return run_dense(p, pl, M, N, C, ldc, accumulate, &nd->st, stream);
+}
