@@ -27,7 +27,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2506_11728_b200 import inputs  # noqa: E402  (bytes only, no arithmetic)
+from paper_2506_11728_b200 import inputs, sharding  # noqa: E402  (bytes / bookkeeping only, no arithmetic)
 
 NOMINAL_INT8_TOPS = 4500.0
 NOMINAL_BF16_TFLOPS = 2250.0
@@ -435,7 +435,8 @@ def main():
         dist.barrier()
     launches = (kernels_per_step * args.steps) if graph is not None else (mg.mipgemm_launch_count() - launches0)
     assert mg.mipgemm_device_status() == mg.OK
-    elapsed_ms = ev0.elapsed_time(ev1)
+    elapsed_ms = sharding.max_over_ranks(ev0.elapsed_time(ev1), dist if world > 1 else None,
+                                         torch.device("cuda", local_rank))
     # per-problem durations (still inside the clock-sampled region)
     detail_reps = 3 if graph is not None else args.steps
     if graph is not None:
@@ -450,11 +451,6 @@ def main():
                 group_ms[j] += a.elapsed_time(b)
     sampler.stop_flag.set()
     sampler.join(timeout=2.0)
-    if world > 1:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
-
     step_ops = sum(p.ops * r for (p, r) in groups)
     step_bytes = sum(p.bytes * r for (p, r) in groups)
     ms_per_step = elapsed_ms / args.steps
