@@ -21,6 +21,7 @@ struct Tuning {
     int block_n = 0, stages = 0, split_k = 0, force_path = 0;
 };
 Tuning g_tuning;
+bool g_tuning_no_cluster_split = false;  // MIPGEMM_NO_CLUSTER_SPLIT=1: split-K through zero fill + TMA reduce-add
 bool g_tuning_no_tma_store = false;   // MIPGEMM_DIRECT_STORE=1: force the direct-store epilogue
 std::atomic<uint64_t> g_launches{0};
 
@@ -86,6 +87,7 @@ int get_device(DeviceState** out) {
             if ((e = dense_init()) != cudaSuccess) return cuda_fail(e);
             d.pair_clusters = dense_pair_max_clusters(kSmemBudget);
             if (const char* ds = std::getenv("MIPGEMM_DIRECT_STORE")) g_tuning_no_tma_store = std::atoi(ds) != 0;
+            if (const char* cs = std::getenv("MIPGEMM_NO_CLUSTER_SPLIT")) g_tuning_no_cluster_split = std::atoi(cs) != 0;
             if ((e = cudaMalloc(&d.status_word, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaMemset(d.status_word, 0, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
             d.status = MIPGEMM_OK;
@@ -190,40 +192,82 @@ uint32_t pow2_at_least(uint32_t v) {
 
 // Tile width, pipeline depth and split-K for an M x N x K problem (k-block = block_k bytes).
 struct Plan {
+    int cluster_split;   // > 1: split_k CTAs of a tile form a cluster and reduce through DSMEM
     int pair;   // 1: CTA pairs share 256-row tiles (cta_group::2)
     int block_n, stages, split_k, kb_per_split, k_blocks, tiles_m, tiles_n;
 };
+
+// Cost model behind the plan (clocks, calibrated on B200 with CUDA-graph timings of this
+// kernel).  One 128-byte k-block of a 128 x bn tile costs what the slower of the tensor pipe
+// (2*bn clk) and the SM's ~64 B/clk ingest from L2 allows; CTA pairs stage only half of B per
+// CTA.  The epilogue of a tile (350 clk per 32-column chunk) hides behind the next tile's main
+// loop; only the last one is exposed.  A launch carries ~3.7 us of fixed cost (launch gap,
+// set-up, pipeline fill, store drain); the DSMEM exchange of a cluster split-K costs about
+// 2.5 / 6 / 13 us for 2 / 4 / 8 CTAs (measured), so it only pays for K-heavy, tile-poor shapes.
+double plan_cost_us(int pair, int bn, int split, long long M, long long N, int k_blocks, int block_k,
+                    const DeviceState* dev) {
+    const double scale = block_k / 128.0;
+    const double kb_clk = (pair ? 300.0 + 1.5 * bn : 250.0 + 2.0 * bn) * scale;
+    const double epi_clk = 350.0 * (bn / 32);
+    const long long rows = pair ? 2 * kBlockM : kBlockM;
+    const long long tiles = ((M + rows - 1) / rows) * ((N + bn - 1) / bn);
+    const long long slots = pair ? dev->pair_clusters : dev->sm_count;
+    const double main = static_cast<double>((k_blocks + split - 1) / split) * kb_clk;
+    double clk;
+    if (split > 1) {
+        const double exchange_us = split == 2 ? 2.5 : (split == 4 ? 6.0 : 13.0);
+        clk = main + epi_clk / split + exchange_us * 1900.0;
+    } else {
+        const long long waves = (tiles + slots - 1) / slots;
+        clk = static_cast<double>(waves - 1) * (main > epi_clk ? main : epi_clk) + main + epi_clk;
+    }
+    return 3.7 + (pair ? 1.0 : 0.0) + clk / 1900.0;   // pairs: cluster launch, two cluster barriers
+}
 
 Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceState* dev) {
     const int sm_count = dev->sm_count;
     Plan pl{};
     pl.k_blocks = static_cast<int>((K + block_k - 1) / block_k);
-    // CTA pairs pay off when there is at least a full wave of 256 x 256 tiles.
-    const long long pair_tiles = ((M + 2 * kBlockM - 1) / (2 * kBlockM)) * ((N + 255) / 256);
-    pl.pair = (dev->pair_clusters > 0 && pair_tiles >= dev->pair_clusters && !g_tuning.block_n) ? 1 : 0;
-    if (g_tuning.force_path == MIPGEMM_PATH_DENSE_PAIR && dev->pair_clusters > 0) pl.pair = 1;
-    if (g_tuning.force_path == MIPGEMM_PATH_DENSE) pl.pair = 0;
+
+    // Candidates: one CTA per tile or CTA pairs, bn in {64, 128, 256}, optionally a cluster
+    // split-K of 2/4/8 when the tiles alone would leave most SMs idle.  Experiment overrides
+    // (mipgemm_set_tuning) restrict the candidate set.
+    int best_pair = 0, best_bn = g_tuning.block_n ? g_tuning.block_n : 128, best_split = 1;
+    double best = 1e30;
+    const bool explicit_split = g_tuning.split_k != 0;
+    for (int pair = 0; pair <= 1; ++pair) {
+        if (pair && dev->pair_clusters <= 0) continue;
+        if (g_tuning.force_path == MIPGEMM_PATH_DENSE_PAIR && !pair && dev->pair_clusters > 0) continue;
+        if (g_tuning.force_path == MIPGEMM_PATH_DENSE && pair) continue;
+        for (int bn = 64; bn <= 256; bn *= 2) {
+            int bn_use = bn;
+            if (g_tuning.block_n) {
+                if (bn != 64) continue;                       // a single candidate: the forced width
+                bn_use = g_tuning.block_n;
+                if (pair && bn_use % 64 != 0) bn_use = (bn_use + 63) / 64 * 64;
+            }
+            const long long rows = pair ? 2 * kBlockM : kBlockM;
+            const long long tiles = ((M + rows - 1) / rows) * ((N + bn_use - 1) / bn_use);
+            for (int split = 1; split <= 8; split *= 2) {
+                if (split > 1) {
+                    if (pair || explicit_split || g_tuning_no_cluster_split) break;
+                    if (tiles * split > sm_count || bn_use / split < 32 || (bn_use / split) % 32 != 0) break;
+                    if (pl.k_blocks / split < 2) break;
+                }
+                const double us = plan_cost_us(pair, bn_use, split, M, N, pl.k_blocks, block_k, dev);
+                if (us < best) {
+                    best = us;
+                    best_pair = pair;
+                    best_bn = bn_use;
+                    best_split = split;
+                }
+            }
+        }
+    }
+    pl.pair = best_pair;
+    const int bn = best_bn;
     const int rows_per_tile = pl.pair ? 2 * kBlockM : kBlockM;
     pl.tiles_m = static_cast<int>((M + rows_per_tile - 1) / rows_per_tile);
-    auto tiles_for = [&](int bn) { return static_cast<long long>(pl.tiles_m) * ((N + bn - 1) / bn); };
-    int bn;
-    if (g_tuning.block_n) {
-        bn = g_tuning.block_n;
-        if (pl.pair && bn % 64 != 0) bn = (bn + 63) / 64 * 64;
-    } else if (pl.pair) {
-        bn = 256;
-    } else if (N <= 64) {
-        bn = 64;
-    } else if (N <= 128) {
-        bn = 128;
-    } else if (tiles_for(256) >= sm_count) {
-        bn = 256;
-    } else if (tiles_for(128) >= sm_count || N <= 256 + 128) {
-        bn = 128;
-    } else {
-        bn = 64;
-        if (tiles_for(64) < sm_count) bn = 128;   // too few tiles either way: prefer the wider MMA, split K
-    }
     pl.block_n = bn;
     pl.tiles_n = static_cast<int>((N + bn - 1) / bn);
     const int stage_bytes = kBlockM * block_k + (pl.pair ? bn / 2 : bn) * block_k;
@@ -232,19 +276,25 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
     if (g_tuning.stages) stages = g_tuning.stages < stages ? g_tuning.stages : stages;
     if (stages < 2) stages = 2;
     pl.stages = stages;
-    int split = 1;
-    const long long tiles = static_cast<long long>(pl.tiles_m) * pl.tiles_n;
-    if (g_tuning.split_k) {
-        split = g_tuning.split_k;
-    } else if (!pl.pair && tiles * 2 <= sm_count && pl.k_blocks >= 8) {
-        split = static_cast<int>(sm_count / tiles);
-        const int max_split = pl.k_blocks / 4;
-        if (split > max_split) split = max_split;
-    }
+
+    int split = explicit_split ? g_tuning.split_k : best_split;
+    if (pl.pair) split = 1;
     if (split > pl.k_blocks) split = pl.k_blocks;
     if (split < 1) split = 1;
+    // the automatic split is a cluster split (DSMEM reduce-scatter: the receive buffers must fit
+    // the idle pipeline stages); an explicit factor uses zero fill + TMA tile reduce-add
+    pl.cluster_split = 0;
+    if (!explicit_split && split > 1) {
+        if (512LL * bn * (split - 1) / split <= static_cast<long long>(stages) * stage_bytes) pl.cluster_split = split;
+        else split = 1;
+    }
     pl.kb_per_split = (pl.k_blocks + split - 1) / split;
     pl.split_k = (pl.k_blocks + pl.kb_per_split - 1) / pl.kb_per_split;
+    if (pl.cluster_split && pl.split_k != pl.cluster_split) {   // a share would be empty: no split
+        pl.cluster_split = 0;
+        pl.split_k = 1;
+        pl.kb_per_split = pl.k_blocks;
+    }
     return pl;
 }
 
@@ -262,8 +312,9 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
     p.tiles_n = pl.tiles_n;
     p.split_k = pl.split_k;
     p.kb_per_split = pl.kb_per_split;
+    p.cluster_split = pl.cluster_split;
     p.group_n = 8;
-    p.use_red = pl.split_k > 1 ? 1 : 0;
+    p.use_red = (pl.split_k > 1 && !pl.cluster_split) ? 1 : 0;
     p.accumulate = p.use_red ? 0 : (accumulate ? 1 : 0);
     const uintptr_t c_addr = reinterpret_cast<uintptr_t>(C);
     p.store_vec = (c_addr % 32 == 0 && ldc % 8 == 0) ? 8 : ((c_addr % 16 == 0 && ldc % 4 == 0) ? 4 : 1);
@@ -275,7 +326,7 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
     // shared memory, and split-K partial tiles are added into C by TMA tile reduce-adds.
     p.c_mode = 0;
     if (c_addr % 16 == 0 && ldc % 4 == 0 && !g_tuning_no_tma_store) {
-        if (pl.split_k > 1) {
+        if (pl.split_k > 1 && !pl.cluster_split) {
             p.c_mode = 2;
             p.use_red = 0;
         } else {
@@ -295,7 +346,7 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
 
 int run_dense(DenseParams& p, const Plan& pl, long long M, long long N, int32_t* C, long long ldc,
               int accumulate, DeviceState* dev, cudaStream_t stream) {
-    if (pl.split_k > 1 && !accumulate) {
+    if (pl.split_k > 1 && !pl.cluster_split && !accumulate) {
         cudaError_t e = launch_fill_zero(C, ldc, M, N, stream);
         ++g_launches;
         if (e != cudaSuccess) return cuda_fail(e);
@@ -321,6 +372,8 @@ int run_dense(DenseParams& p, const Plan& pl, long long M, long long N, int32_t*
     if (pl.pair) {
         const int clusters = static_cast<int>(units < dev->pair_clusters ? units : dev->pair_clusters);
         e = launch_dense_pair(p, 2 * clusters, smem, stream);
+    } else if (pl.cluster_split) {
+        e = launch_dense_cluster(p, static_cast<int>(units), pl.cluster_split, smem, stream);
     } else {
         const int grid = static_cast<int>(units < dev->sm_count ? units : dev->sm_count);
         e = launch_dense(p, grid, smem, stream);

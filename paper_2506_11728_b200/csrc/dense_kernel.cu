@@ -30,10 +30,7 @@ namespace mip {
 
 #ifdef MIPGEMM_TRACE
 #define MIP_STAMP(slot) do { if (p.trace && blockIdx.x == 0 && (threadIdx.x & 31) == 0) p.trace[slot] = globaltimer_ns(); } while (0)
-__shared__ long long mip_trace_smem[32];
-#define MIP_CLK(slot) do { if (blockIdx.x == 0 && threadIdx.x == 64 && mip_trace_smem[slot] == 0) mip_trace_smem[slot] = clock64(); } while (0)
 #else
-#define MIP_CLK(slot) do { } while (0)
 #define MIP_STAMP(slot) do { } while (0)
 #endif
 
@@ -43,8 +40,9 @@ struct TileCoord {
 
 __device__ __forceinline__ TileCoord decode_unit(const DenseParams& p, int unit, int rows_per_tile) {
     const int tiles_mn = p.tiles_m * p.tiles_n;
-    const int ks = unit / tiles_mn;
-    const int t = unit - ks * tiles_mn;
+    // cluster split-K: the CTAs of a cluster (consecutive units) share one tile
+    const int ks = p.cluster_split > 1 ? unit % p.cluster_split : unit / tiles_mn;
+    const int t = p.cluster_split > 1 ? unit / p.cluster_split : unit - ks * tiles_mn;
     // Rasterisation: groups of `group_n` tile columns are swept top to bottom with the
     // column index fastest, so the B panel of a group stays in L2 while A streams by.
     const int per_group = p.group_n * p.tiles_m;
@@ -146,15 +144,11 @@ __device__ __forceinline__ void tma_store_slab(const DenseParams& p, uint32_t bu
 // base and ldc % 4 == 0.  (row0, col0) is the chunk's origin in C.
 __device__ __forceinline__ void coalesced_chunk(const DenseParams& p, uint32_t buf, const uint32_t (&v)[32],
                                                 int lane, int row0, int col0) {
-    MIP_CLK(24);
     __syncwarp();   // the previous chunk's reads of `buf` are done
-    MIP_CLK(25);
     const uint32_t mine = buf + static_cast<uint32_t>(lane) * 128u;
 #pragma unroll
     for (int j = 0; j < 8; ++j) st_shared_v4(mine + (static_cast<uint32_t>(j ^ (lane & 7)) << 4), &v[4 * j]);
-    MIP_CLK(26);
     __syncwarp();
-    MIP_CLK(27);
     const int piece = lane & 7;                 // which 16 bytes (4 columns) of a row
     const int col = col0 + 4 * piece;
     const int cols_left = p.N - col;            // <= 0: nothing of this piece is inside C
@@ -212,9 +206,6 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
     const int unit_stride = kPair ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
     const int b_rows = kPair ? (p.block_n >> 1) : p.block_n;   // rows of B staged by this CTA
     MIP_STAMP(0);
-#ifdef MIPGEMM_TRACE
-    if (threadIdx.x < 32) mip_trace_smem[threadIdx.x] = 0;
-#endif
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t pad = ((raw_addr + 1023u) & ~1023u) - raw_addr;
@@ -425,34 +416,30 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             const uint32_t acc = t & 1, acc_phase = (t >> 1) & 1;
             if (!mbar_wait(bar_tfull + 8u * acc, acc_phase, abort_flag, budget)) break;
             if (t == 0 && warp == 2) MIP_STAMP(5);
-            MIP_CLK(20);
             tc_fence_after();
             const int m_cta = tc.m0 + static_cast<int>(cta_rank) * kBlockM;
             const int row = m_cta + q * 32 + lane;
             const int n_rem = p.N - tc.n0;
             const int n_here = min(p.block_n, n_rem);
-            if (p.c_mode == 1 || m_cta + q * 32 < p.M) {   // (slab stores need all four warps)
+            if (p.cluster_split > 1) {
+                // the accumulator stays in tensor memory; the cluster reduces it below
+            } else if (p.c_mode == 1 || m_cta + q * 32 < p.M) {   // (slab stores need all four warps)
                 int32_t* crow = p.C + static_cast<long long>(row) * p.ldc + tc.n0;
                 const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.block_n;
                 const uint32_t my_staging = staging + static_cast<uint32_t>(q) * 8192u;
                 // two register buffers: the TMEM load of the next chunk is in flight while the
                 // current one is written out
                 uint32_t va[32], vb[32];
-                MIP_CLK(21);
                 tmem_ld_32x32(t_row, va);
-                MIP_CLK(22);
                 for (int c0 = 0; c0 < n_here; c0 += 64) {
                     tmem_ld_wait();
-                    MIP_CLK(23);
                     if (c0 + 32 < n_here) tmem_ld_32x32(t_row + c0 + 32, vb);
                     if (p.c_mode == 1) tma_store_slab(p, staging, va, lane, q, warp == 2, tc.n0 + c0, m_cta);
                     else if (p.c_mode == 3) coalesced_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0);
                     else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging, va, lane, tc.n0 + c0, m_cta + q * 32);
                     else if (row < p.M) store_chunk(p, crow + c0, va, min(32, n_here - c0));
-                    MIP_CLK(28);
                     if (c0 + 32 < n_here) {
                         tmem_ld_wait();
-                        MIP_CLK(29);
                         if (c0 + 64 < n_here) tmem_ld_32x32(t_row + c0 + 64, va);
                         if (p.c_mode == 1) tma_store_slab(p, staging + 16384u, vb, lane, q, warp == 2, tc.n0 + c0 + 32, m_cta);
                         else if (p.c_mode == 3) coalesced_chunk(p, my_staging + 4096u, vb, lane, m_cta + q * 32, tc.n0 + c0 + 32);
@@ -461,7 +448,6 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     }
                 }
             }
-            MIP_CLK(30);
             if (warp == 2) { if (t == 0) MIP_STAMP(6); MIP_STAMP(7); }
             tc_fence_before();
             __syncwarp();
@@ -471,7 +457,79 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             }
         }
         // every tile copy issued by this warp must be complete before the CTA may exit
-        if ((p.c_mode == 2 || (p.c_mode == 1 && warp == 2)) && elect_one()) tma_store_wait<0>();
+        if (p.cluster_split <= 1 && (p.c_mode == 2 || (p.c_mode == 1 && warp == 2)) && elect_one())
+            tma_store_wait<0>();
+    }
+
+    if (!kPair && p.cluster_split > 1) {
+        // ---------------------------------------------------------------- cluster split-K
+        // The S CTAs of a cluster hold partial sums of the same tile (one K share each) in
+        // their tensor memories.  Reduce-scatter through distributed shared memory: CTA r owns
+        // the r-th slice of the tile's columns; every CTA sends its partial of slice d to CTA
+        // d, which adds the S partials (exact integer adds, any order) and stores its slice.
+        // The receive buffers alias the pipeline stages, hence the first cluster barrier: it
+        // completes only when every CTA's epilogue warps have seen their accumulator ready,
+        // i.e. when no MMA in the cluster can still read stage memory.
+        const uint32_t S = static_cast<uint32_t>(p.cluster_split);
+        const uint32_t rank = cluster_ctarank();
+        const int slice_cols = p.block_n / static_cast<int>(S);
+        const int chunks = slice_cols >> 5;
+        const int q = warp & 3;
+        const int r_tile = q * 32 + lane;                       // this thread's row of the tile
+        const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+        const TileCoord tc = decode_unit(p, first_unit, kRowsPerTile);
+        tc_fence_before();
+        cluster_arrive();
+        cluster_wait();
+        tc_fence_after();
+        if (warp >= 2 && *abort_flag == 0) {
+            for (uint32_t d = 0; d < S; ++d) {
+                if (d == rank) continue;
+                const uint32_t slot = rank < d ? rank : rank - 1;            // my slot among d's S-1 senders
+                for (int c = 0; c < chunks; ++c) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(t_row + d * slice_cols + c * 32, v);
+                    tmem_ld_wait();
+                    const uint32_t local = smem_base + ((slot * chunks + c) * 128u + r_tile) * 128u;
+                    const uint32_t remote = mapa_u32(local, d);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};"
+                                     ::"r"(remote + (static_cast<uint32_t>(j ^ (r_tile & 7)) << 4)), "r"(v[4 * j]),
+                                       "r"(v[4 * j + 1]), "r"(v[4 * j + 2]), "r"(v[4 * j + 3]) : "memory");
+                }
+            }
+        }
+        cluster_arrive();
+        cluster_wait();
+        if (warp >= 2 && *abort_flag == 0) {
+            const int m_cta = tc.m0;
+            const int row = m_cta + r_tile;
+            const uint32_t my_staging = staging + static_cast<uint32_t>(q) * 8192u;
+            for (int c = 0; c < chunks; ++c) {
+                const int col0 = tc.n0 + static_cast<int>(rank) * slice_cols + c * 32;
+                if (col0 >= p.N) break;                                     // uniform over the CTA
+                uint32_t v[32];
+                tmem_ld_32x32(t_row + rank * slice_cols + c * 32, v);
+                tmem_ld_wait();
+                for (uint32_t slot = 0; slot + 1 < S; ++slot) {
+                    const uint32_t src = smem_base + ((slot * chunks + c) * 128u + r_tile) * 128u;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        uint32_t x[4];
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
+                                     : "r"(src + (static_cast<uint32_t>(j ^ (r_tile & 7)) << 4)) : "memory");
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) v[4 * j + e] += x[e];
+                    }
+                }
+                if (p.c_mode == 1) tma_store_slab(p, staging + (c & 1) * 16384u, v, lane, q, warp == 2, col0, m_cta);
+                else if (p.c_mode == 3) coalesced_chunk(p, my_staging + (c & 1) * 4096u, v, lane, m_cta + q * 32, col0);
+                else if (row < p.M) store_chunk(p, p.C + static_cast<long long>(row) * p.ldc + col0, v, min(32, p.N - col0));
+            }
+            if (p.c_mode == 1 && warp == 2 && elect_one()) tma_store_wait<0>();
+        }
     }
 
     tc_fence_before();
@@ -486,9 +544,6 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         tmem_dealloc<kGroup>(tmem_base, p.tmem_cols);
     }
     if (threadIdx.x == 0) MIP_STAMP(9);
-#ifdef MIPGEMM_TRACE
-    if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) for (int i = 20; i < 32; ++i) p.trace[i] = mip_trace_smem[i];
-#endif
     if (threadIdx.x == 0 && *abort_flag != 0) atomicOr(p.status, 1u);
 }
 
@@ -503,6 +558,25 @@ cudaError_t dense_init() {
 cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream) {
     mip_dense_kernel<false><<<grid, kDenseThreads, smem_bytes, stream>>>(p);
     return cudaGetLastError();
+}
+
+// One-CTA-per-tile kernel launched in clusters of `cluster` CTAs (cluster split-K); `grid` is a
+// multiple of `cluster`.
+cudaError_t launch_dense_cluster(const DenseParams& p, int grid, int cluster, size_t smem_bytes,
+                                 cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+    cfg.blockDim = dim3(kDenseThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false>, p);
 }
 
 // `grid` counts CTAs and must be even: consecutive CTAs form a cluster of two.

@@ -32,6 +32,7 @@ struct alignas(64) DenseParams {
     int stages;
     int tiles_m, tiles_n;
     int split_k, kb_per_split;
+    int cluster_split;       // > 1: the split_k CTAs sharing a tile form a cluster and reduce through DSMEM
     int group_n;             // n-tiles per rasterisation group
     int accumulate;          // epilogue adds the incoming C
     int use_red;             // epilogue reduces with red.global.add (split-K)
@@ -51,6 +52,7 @@ struct alignas(64) DenseParams {
 };
 
 cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream);
+cudaError_t launch_dense_cluster(const DenseParams& p, int grid, int cluster, size_t smem_bytes, cudaStream_t stream);
 cudaError_t launch_dense_pair(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream);
 int dense_pair_max_clusters(size_t smem_bytes);
 cudaError_t dense_init();  // opt in to large dynamic shared memory (once per device)
