@@ -22,6 +22,7 @@ struct Tuning {
 };
 Tuning g_tuning;
 bool g_tuning_no_cluster_split = false;  // MIPGEMM_NO_CLUSTER_SPLIT=1: split-K through zero fill + TMA reduce-add
+bool g_tuning_no_skinny_ring = false;    // MIPGEMM_NO_SKINNY_RING=1: always the register form of the skinny kernel
 bool g_tuning_no_tma_store = false;   // MIPGEMM_DIRECT_STORE=1: force the direct-store epilogue
 std::atomic<uint64_t> g_launches{0};
 
@@ -88,6 +89,7 @@ int get_device(DeviceState** out) {
             d.pair_clusters = dense_pair_max_clusters(kSmemBudget);
             if (const char* ds = std::getenv("MIPGEMM_DIRECT_STORE")) g_tuning_no_tma_store = std::atoi(ds) != 0;
             if (const char* cs = std::getenv("MIPGEMM_NO_CLUSTER_SPLIT")) g_tuning_no_cluster_split = std::atoi(cs) != 0;
+            if (const char* sr = std::getenv("MIPGEMM_NO_SKINNY_RING")) g_tuning_no_skinny_ring = std::atoi(sr) != 0;
             if ((e = cudaMalloc(&d.status_word, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaMemset(d.status_word, 0, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
             d.status = MIPGEMM_OK;
@@ -428,6 +430,31 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     if (M <= 16 && g_tuning.force_path != MIPGEMM_PATH_DENSE && g_tuning.force_path != MIPGEMM_PATH_DENSE_PAIR) {
         SkinnyParams sp{A, lda, B, ldb, C, ldc, static_cast<int>(M), static_cast<int>(N),
                         static_cast<int>(K), a_unsigned ? 1 : 0, accumulate ? 1 : 0};
+        if (skinny_ring_supported(sp, dev->sm_count) && !g_tuning_no_skinny_ring) {
+            SkinnyRingParams rp;
+            std::memset(&rp, 0, sizeof(rp));
+            cuuint64_t dims[3] = {128, static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(K / 128)};
+            cuuint64_t strides[2] = {static_cast<cuuint64_t>(ldb), 128};
+            cuuint32_t box[3] = {128, 16, 8};
+            cuuint32_t estr[3] = {1, 1, 1};
+            CUresult r = g_encode_tiled(&rp.tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(B), dims,
+                                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r == CUDA_SUCCESS) {   // (a driver that refuses the overlapping strides: register form below)
+                rp.A = A; rp.lda = lda; rp.C = C; rp.ldc = ldc;
+                rp.M = static_cast<int>(M); rp.N = static_cast<int>(N); rp.K = static_cast<int>(K);
+                rp.a_unsigned = a_unsigned ? 1 : 0; rp.accumulate = accumulate ? 1 : 0;
+                rp.status = dev->status_word;
+                rp.wait_budget_ns = 4000000000ull;
+                cudaError_t e = launch_skinny_ring(rp, dev->sm_count, stream);
+                ++g_launches;
+                if (e != cudaSuccess) return cuda_fail(e);
+                tl_last_path = MIPGEMM_PATH_SKINNY | path_flags;
+                return MIPGEMM_OK;
+            }
+            tl_last_cuda_error = 100000 + static_cast<int>(r);
+        }
         if (skinny_supported(sp)) {
             cudaError_t e = launch_skinny(sp, stream);
             ++g_launches;

@@ -68,6 +68,20 @@ struct SkinnyParams {
 cudaError_t launch_skinny(const SkinnyParams& p, cudaStream_t stream);
 bool skinny_supported(const SkinnyParams& p);
 
+// Ring form of the skinny kernel (weights streamed through a TMA-fed shared-memory ring).
+struct alignas(64) SkinnyRingParams {
+    CUtensorMap tmap_b;      // rank-3 byte tensor {128, N, K/128}, strides {ldb, 128}, box {128, 16, 8}
+    const void* A; long long lda;
+    int32_t* C; long long ldc;
+    int M, N, K;
+    int a_unsigned, accumulate;
+    int slots, tokens_in_smem;   // filled in by the launcher
+    unsigned int* status;
+    unsigned long long wait_budget_ns;
+};
+bool skinny_ring_supported(const SkinnyParams& p, int sm_count);
+cudaError_t launch_skinny_ring(const SkinnyRingParams& p, int sm_count, cudaStream_t stream);
+
 // Auxiliary kernels.
 cudaError_t launch_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,
                           long long rows, long long cols, cudaStream_t stream);
