@@ -261,6 +261,11 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         cluster_wait();
     }
     tc_fence_after();
+    // Programmatic dependent launch: everything so far touched only shared memory, tensor memory
+    // and kernel parameters and may overlap the tail of the previous kernel in the stream; from
+    // here on global memory is read and written, which must wait for that kernel to finish.
+    pdl_launch_dependents();
+    pdl_wait();
     const uint32_t tmem_base = *tmem_slot;
     if (threadIdx.x == 0) MIP_STAMP(1);
 
@@ -555,9 +560,23 @@ cudaError_t dense_init() {
                                 kSmemBudget);
 }
 
+// All launches allow programmatic stream serialisation (see pdl_wait() in the kernel).
+static void pdl_attribute(cudaLaunchAttribute& a) {
+    a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    a.val.programmaticStreamSerializationAllowed = 1;
+}
+
 cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream) {
-    mip_dense_kernel<false><<<grid, kDenseThreads, smem_bytes, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+    cfg.blockDim = dim3(kDenseThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    pdl_attribute(attr[0]);
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false>, p);
 }
 
 // One-CTA-per-tile kernel launched in clusters of `cluster` CTAs (cluster split-K); `grid` is a
@@ -569,13 +588,14 @@ cudaError_t launch_dense_cluster(const DenseParams& p, int grid, int cluster, si
     cfg.blockDim = dim3(kDenseThreads, 1, 1);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = static_cast<unsigned>(cluster);
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    pdl_attribute(attr[1]);
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false>, p);
 }
 
@@ -586,13 +606,14 @@ cudaError_t launch_dense_pair(const DenseParams& p, int grid, size_t smem_bytes,
     cfg.blockDim = dim3(kDenseThreads, 1, 1);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    pdl_attribute(attr[1]);
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true>, p);
 }
 

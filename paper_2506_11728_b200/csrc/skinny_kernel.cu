@@ -112,6 +112,8 @@ mip_skinny_kernel(const SkinnyParams p, int split) {
     constexpr int kDepth = MIP_SKINNY_DEPTH;   // slices in flight per warp
     __shared__ int red[kSkinnyWarps][16][17];        // per-warp partials [weight row][token]
     __shared__ int gather[kSkinnyMaxSplit][256];     // rank 0 only: per-CTA partials of the cluster
+    pdl_launch_dependents();   // (programmatic dependent launch: see ptx.cuh)
+    pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
     const uint32_t rank = split > 1 ? cluster_ctarank() : 0u;
@@ -218,13 +220,15 @@ static cudaError_t launch_skinny_t(const SkinnyParams& p, int split, cudaStream_
     cfg.blockDim = dim3(kSkinnyWarps * 32, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = static_cast<unsigned>(split);
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, mip_skinny_kernel<kU, kTwo>, p, split);
 }
 

@@ -133,6 +133,10 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
         fence_mbar_init();
         tma_prefetch_desc(&p.tmap_b);
     }
+    // Everything above touched only shared memory and kernel parameters, so it may overlap the
+    // tail of the previous kernel in the stream; nothing below may.
+    pdl_launch_dependents();
+    pdl_wait();
     __syncthreads();
 
     const int units = (p.N + 15) >> 4;
@@ -269,8 +273,17 @@ cudaError_t launch_ring_t(SkinnyRingParams p, int grid, cudaStream_t stream) {
     if (slots > kMaxRingSlots) slots = kMaxRingSlots;
     p.slots = slots;
     const size_t smem = static_cast<size_t>(slots) * kSlotBytes + fixed + (p.tokens_in_smem ? tok_bytes : 0);
-    mip_skinny_ring_kernel<kU, kTwo><<<grid, kRingThreads, smem, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+    cfg.blockDim = dim3(kRingThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, mip_skinny_ring_kernel<kU, kTwo>, p);
 }
 
 }  // namespace
