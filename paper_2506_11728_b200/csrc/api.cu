@@ -86,6 +86,7 @@ int get_device(DeviceState** out) {
                 g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(fn);
             }
             if ((e = dense_init()) != cudaSuccess) return cuda_fail(e);
+            if ((e = skinny_ring_init()) != cudaSuccess) return cuda_fail(e);
             d.pair_clusters = dense_pair_max_clusters(kSmemBudget);
             if (const char* ds = std::getenv("MIPGEMM_DIRECT_STORE")) g_tuning_no_tma_store = std::atoi(ds) != 0;
             if (const char* cs = std::getenv("MIPGEMM_NO_CLUSTER_SPLIT")) g_tuning_no_cluster_split = std::atoi(cs) != 0;

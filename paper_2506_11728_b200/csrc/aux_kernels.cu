@@ -292,13 +292,10 @@ __global__ void __launch_bounds__(128, 1) mip_probe_kernel(int iters, int32_t* s
 
 cudaError_t launch_probe(int iters, int grid, int32_t* sink, cudaStream_t stream) {
     const size_t smem = 128 * 128 + 256 * 128 + 64 + 1024;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(mip_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(smem));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    // (set on every launch: the attribute is per device and the probe is not a hot path)
+    cudaError_t e = cudaFuncSetAttribute(mip_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
     mip_probe_kernel<<<grid, 128, smem, stream>>>(iters, sink);
     return cudaGetLastError();
 }

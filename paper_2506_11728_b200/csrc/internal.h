@@ -80,6 +80,7 @@ struct alignas(64) SkinnyRingParams {
     unsigned long long wait_budget_ns;
 };
 bool skinny_ring_supported(const SkinnyParams& p, int sm_count);
+cudaError_t skinny_ring_init();  // once per device
 cudaError_t launch_skinny_ring(const SkinnyRingParams& p, int sm_count, cudaStream_t stream);
 
 // Auxiliary kernels.

@@ -258,13 +258,6 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
 
 template <bool kU, bool kTwo>
 cudaError_t launch_ring_t(SkinnyRingParams p, int grid, cudaStream_t stream) {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(mip_skinny_ring_kernel<kU, kTwo>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmemMax);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
     // tokens move into shared memory when they leave room for at least 6 ring slots
     const int fixed = kRedBytes + kRingCtrlBytes + 1024;
     const int tok_bytes = p.M * (p.K + kTokenPad);
@@ -287,6 +280,19 @@ cudaError_t launch_ring_t(SkinnyRingParams p, int grid, cudaStream_t stream) {
 }
 
 }  // namespace
+
+// Opt in to large dynamic shared memory for the current device (once per device).
+cudaError_t skinny_ring_init() {
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(mip_skinny_ring_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  kRingSmemMax)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(mip_skinny_ring_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  kRingSmemMax)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(mip_skinny_ring_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  kRingSmemMax)) != cudaSuccess) return e;
+    return cudaFuncSetAttribute(mip_skinny_ring_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                kRingSmemMax);
+}
 
 bool skinny_ring_supported(const SkinnyParams& p, int sm_count) {
     if (!skinny_supported(p)) return false;
