@@ -31,6 +31,8 @@
  *
  * where a term whose input row or column falls outside the image contributes 0.
  *
+ * Dequantised results: mip_oracle_dequant (definition C^r = s * C^q in binary64).
+ *
  * Pins: tests/test_oracle_pins.py (brute force on tiny inputs, closed forms,
  * extremes, range check, checksum identities, NumPy integer matmul, conv vs
  * explicit im2col, shifted-copy filters).
@@ -140,6 +142,19 @@ int64_t mip_oracle_conv(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t C
         }
     }
     return overflow_cells;
+}
+
+/*
+ * Dequantisation of an integer result (paper, Section 7.3: C^r = s_A s_B C^q): every exact integer
+ * sum is multiplied by the scale as a real number, here in binary64 (the product of a 32-bit
+ * integer and a binary32 scale is exact in binary64: 31 + 24 significant bits).  The GPU path
+ * rounds to binary32 twice (conversion, multiplication); tests allow the 2^-23 relative error
+ * that follows from that.
+ */
+void mip_oracle_dequant(const int32_t *Cq, int64_t count, double scale, double *Cr)
+{
+    for (int64_t i = 0; i < count; ++i)
+        Cr[i] = scale * (double)Cq[i];
 }
 
 #ifdef _OPENMP

@@ -47,6 +47,8 @@ def _load():
         lib.mip_oracle_gemm.argtypes = [ci, i64, i64, i64, vp, i64, vp, i64, vp, i64, ci]
         lib.mip_oracle_conv.restype = i64
         lib.mip_oracle_conv.argtypes = [i64] * 13 + [vp, vp, vp, ci]
+        lib.mip_oracle_dequant.restype = None
+        lib.mip_oracle_dequant.argtypes = [vp, i64, ctypes.c_double, vp]
         lib.mip_oracle_threads.restype = ci
         lib.mip_oracle_threads.argtypes = []
         _lib = lib
@@ -142,3 +144,13 @@ def conv(X: np.ndarray, Wt: np.ndarray, *, stride=(1, 1), pad=(0, 0), dil=(1, 1)
     if rc > 0 and not allow_overflow:
         raise OracleOverflow("%d cells do not fit int32" % rc)
     return Y
+
+
+def dequant(Cq: np.ndarray, scale: float) -> np.ndarray:
+    """C^r = scale * C^q (paper Section 7.3) in binary64, element by element; same shape as Cq."""
+    if Cq.dtype != np.int32:
+        raise TypeError("Cq must be int32")
+    flat = np.ascontiguousarray(Cq).reshape(-1)
+    out = np.empty(flat.size, dtype=np.float64)
+    _load().mip_oracle_dequant(_ptr(flat), flat.size, float(scale), _ptr(out))
+    return out.reshape(Cq.shape)

@@ -292,3 +292,24 @@ def test_inputs_deterministic_and_in_range():
     c = inputs.uniform_s32(5000, 9)
     assert c.min() >= -(1 << 20) and c.max() <= (1 << 20)
     assert sum(x[0] for x in inputs.RESNET50_CONVS) == 53 and len(inputs.RESNET50_CONVS) == 23
+
+
+# ---------------------------------------------------------------------------
+# Dequantisation C^r = s * C^q: closed forms and NumPy's own float64 product.
+# ---------------------------------------------------------------------------
+def test_dequant_closed_forms():
+    Cq = np.array([0, 1, -1, 2147483647, -2147483648, 16777217, -123456789], dtype=np.int32)
+    assert np.array_equal(orc.dequant(Cq, 1.0), Cq.astype(np.float64))
+    assert np.array_equal(orc.dequant(Cq, 0.0), np.zeros(7))
+    assert np.array_equal(orc.dequant(Cq, -0.5), Cq.astype(np.float64) * -0.5)        # power of two: exact
+    assert np.array_equal(orc.dequant(Cq, 2.0 ** -20), Cq.astype(np.float64) / 1048576.0)
+    s = float(np.float32(0.0123))
+    got = orc.dequant(Cq, s)
+    assert np.array_equal(got, np.multiply(Cq.astype(np.float64), s))                 # library product
+    # the product of a 32-bit integer and a binary32 scale is exact in binary64: compare with
+    # exact rational arithmetic
+    from fractions import Fraction
+    for c, g in zip(Cq.tolist(), got.tolist()):
+        assert Fraction(g) == Fraction(c) * Fraction(s)
+    two_d = orc.dequant(Cq[:6].reshape(2, 3), 3.0)
+    assert two_d.shape == (2, 3) and two_d[1, 2] == 3.0 * 16777217
