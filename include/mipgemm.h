@@ -128,6 +128,29 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
                          int accumulate, void *stream);
 
 /*
+ * Fused dequantisation (paper Section 7.3: with A ~ s_A A^q and B ~ s_B B^q, the real-valued
+ * product is approximated by C^r = s_A s_B C^q; the paper applies the scale as a separate, cheap
+ * floating-point step after the integer GEMM).  These entry points compute the same exact int32
+ * sums as the ones above and write  C(float32) = scale * sum  from the epilogue, so C is written
+ * once as float and never exists as int32 in memory.  `scale` is the caller's s_A * s_B.
+ * Rounding (the paper fixes none): the int32 sum is converted to binary32 with round-to-nearest-
+ * even and multiplied by `scale` in binary32 (round-to-nearest-even); the result is therefore
+ * within 2^-23 relative of the real number scale*sum, and bit-identical across kernel paths.
+ * Same layouts, limits and return codes as the int32 entry points; there is no accumulate form.
+ */
+int mipgemm_s8s8f32_dequant(int64_t M, int64_t N, int64_t K,
+                            const int8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                            float *C, int64_t ldc, float scale, void *stream);
+int mipgemm_u8s8f32_dequant(int64_t M, int64_t N, int64_t K,
+                            const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                            float *C, int64_t ldc, float scale, void *stream);
+int mipgemm_conv_u8s8f32_dequant(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout,
+                                 int R, int S, int stride_h, int stride_w,
+                                 int pad_h, int pad_w, int dil_h, int dil_w,
+                                 const uint8_t *X, const int8_t *Wt, float *Y,
+                                 float scale, void *stream);
+
+/*
  * Host-buffer variants (the end-to-end path): A, B and C are HOST pointers (pinned or
  * pageable) with the same layouts as above.  The call stages the operands into device
  * memory obtained with cudaMallocAsync on `stream`, runs the device entry point, copies

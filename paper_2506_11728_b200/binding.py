@@ -35,6 +35,9 @@ SIGNATURES = {
     "mipgemm_s8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_u8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_conv_u8s8s32": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, _int, _vp]),
+    "mipgemm_s8s8f32_dequant": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]),
+    "mipgemm_u8s8f32_dequant": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]),
+    "mipgemm_conv_u8s8f32_dequant": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, ctypes.c_float, _vp]),
     "mipgemm_host_s8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_host_u8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_s8s8s32_static_scratch": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
@@ -104,6 +107,24 @@ def mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, p
     return _check(_lib.mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
                                             dil_h, dil_w, _ptr(X), _ptr(Wt), _ptr(Y),
                                             int(bool(accumulate)), _stream(stream)), check)
+
+
+def mipgemm_s8s8f32_dequant(M, N, K, A, lda, B, ldb, C, ldc, scale, stream=None, check=True) -> int:
+    """C[float32] = scale * (A * B): the exact int32 sum, converted and scaled in the epilogue."""
+    return _check(_lib.mipgemm_s8s8f32_dequant(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                               float(scale), _stream(stream)), check)
+
+
+def mipgemm_u8s8f32_dequant(M, N, K, A, lda, B, ldb, C, ldc, scale, stream=None, check=True) -> int:
+    return _check(_lib.mipgemm_u8s8f32_dequant(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                               float(scale), _stream(stream)), check)
+
+
+def mipgemm_conv_u8s8f32_dequant(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w,
+                                 X, Wt, Y, scale, stream=None, check=True) -> int:
+    return _check(_lib.mipgemm_conv_u8s8f32_dequant(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
+                                                    dil_h, dil_w, _ptr(X), _ptr(Wt), _ptr(Y), float(scale),
+                                                    _stream(stream)), check)
 
 
 def mipgemm_host_s8s8s32(M, N, K, A, lda, B, ldb, C, ldc, accumulate=0, stream=None, check=True) -> int:

@@ -16,6 +16,9 @@ using namespace mip;
 
 thread_local int tl_last_path = MIPGEMM_PATH_NONE;
 thread_local int tl_last_cuda_error = 0;
+// Output transform of the call in progress on this thread (set by the *_dequant entry points).
+thread_local int tl_out_f32 = 0;
+thread_local float tl_out_scale = 1.0f;
 
 struct Tuning {
     int block_n = 0, stages = 0, split_k = 0, force_path = 0;
@@ -237,7 +240,8 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
     // (mipgemm_set_tuning) restrict the candidate set.
     int best_pair = 0, best_bn = g_tuning.block_n ? g_tuning.block_n : 128, best_split = 1;
     double best = 1e30;
-    const bool explicit_split = g_tuning.split_k != 0;
+    // (an explicit split reduces int32 tiles in global memory, which a float output cannot share)
+    const bool explicit_split = g_tuning.split_k != 0 && !tl_out_f32;
     for (int pair = 0; pair <= 1; ++pair) {
         if (pair && dev->pair_clusters <= 0) continue;
         if (g_tuning.force_path == MIPGEMM_PATH_DENSE_PAIR && !pair && dev->pair_clusters > 0) continue;
@@ -337,6 +341,8 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
             if (const char* cm = std::getenv("MIPGEMM_CMODE")) p.c_mode = std::atoi(cm);
         }
     }
+    p.out_f32 = tl_out_f32;
+    p.out_scale = tl_out_scale;
     p.a_im2col = 0;
     p.status = dev->status_word;
     p.wait_budget_ns = 4000000000ull;
@@ -430,7 +436,7 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     // ---- skinny path
     if (M <= 16 && g_tuning.force_path != MIPGEMM_PATH_DENSE && g_tuning.force_path != MIPGEMM_PATH_DENSE_PAIR) {
         SkinnyParams sp{A, lda, B, ldb, C, ldc, static_cast<int>(M), static_cast<int>(N),
-                        static_cast<int>(K), a_unsigned ? 1 : 0, accumulate ? 1 : 0};
+                        static_cast<int>(K), a_unsigned ? 1 : 0, accumulate ? 1 : 0, tl_out_f32, tl_out_scale};
         if (skinny_ring_supported(sp, dev->sm_count) && !g_tuning_no_skinny_ring) {
             SkinnyRingParams rp;
             std::memset(&rp, 0, sizeof(rp));
@@ -446,6 +452,7 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
                 rp.A = A; rp.lda = lda; rp.C = C; rp.ldc = ldc;
                 rp.M = static_cast<int>(M); rp.N = static_cast<int>(N); rp.K = static_cast<int>(K);
                 rp.a_unsigned = a_unsigned ? 1 : 0; rp.accumulate = accumulate ? 1 : 0;
+                rp.out_f32 = tl_out_f32; rp.out_scale = tl_out_scale;
                 rp.status = dev->status_word;
                 rp.wait_budget_ns = 4000000000ull;
                 cudaError_t e = launch_skinny_ring(rp, dev->sm_count, stream);
@@ -725,6 +732,33 @@ int mipgemm_host_s8s8s32(int64_t M, int64_t N, int64_t K, const int8_t* A, int64
 int mipgemm_host_u8s8s32(int64_t M, int64_t N, int64_t K, const uint8_t* A, int64_t lda, const int8_t* B,
                          int64_t ldb, int32_t* C, int64_t ldc, int accumulate, void* stream) {
     return host_impl(true, M, N, K, A, lda, B, ldb, C, ldc, accumulate, stream);
+}
+
+// Fused dequantisation: run the integer entry point with the output transform switched on for
+// this thread.  (float 0.0 and int32 0 share their bit pattern, so the K == 0 zero fill is right.)
+struct OutputTransformScope {
+    OutputTransformScope(float scale) { tl_out_f32 = 1; tl_out_scale = scale; }
+    ~OutputTransformScope() { tl_out_f32 = 0; tl_out_scale = 1.0f; }
+};
+
+int mipgemm_s8s8f32_dequant(int64_t M, int64_t N, int64_t K, const int8_t* A, int64_t lda, const int8_t* B,
+                            int64_t ldb, float* C, int64_t ldc, float scale, void* stream) {
+    OutputTransformScope scope(scale);
+    return gemm_impl(false, M, N, K, A, lda, B, ldb, reinterpret_cast<int32_t*>(C), ldc, 0, stream, 0);
+}
+
+int mipgemm_u8s8f32_dequant(int64_t M, int64_t N, int64_t K, const uint8_t* A, int64_t lda, const int8_t* B,
+                            int64_t ldb, float* C, int64_t ldc, float scale, void* stream) {
+    OutputTransformScope scope(scale);
+    return gemm_impl(true, M, N, K, A, lda, B, ldb, reinterpret_cast<int32_t*>(C), ldc, 0, stream, 0);
+}
+
+int mipgemm_conv_u8s8f32_dequant(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int R, int S,
+                                 int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                                 const uint8_t* X, const int8_t* Wt, float* Y, float scale, void* stream) {
+    OutputTransformScope scope(scale);
+    return mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, X, Wt,
+                                reinterpret_cast<int32_t*>(Y), 0, stream);
 }
 
 uint64_t mipgemm_launch_count(void) { return g_launches.load(); }

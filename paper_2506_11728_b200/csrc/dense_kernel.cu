@@ -60,6 +60,13 @@ __device__ __forceinline__ TileCoord decode_unit(const DenseParams& p, int unit,
     return c;
 }
 
+// Fused dequantisation (paper Section 7.3, C^r = s_A s_B C^q): the exact int32 sum is converted to
+// binary32 (round to nearest even) and multiplied by the scale in binary32.
+__device__ __forceinline__ void dequant_chunk(const DenseParams& p, uint32_t (&v)[32]) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__int2float_rn(static_cast<int>(v[j])) * p.out_scale);
+}
+
 // Writes one 32-column chunk of one row of the tile.
 __device__ __forceinline__ void store_chunk(const DenseParams& p, int32_t* dst, uint32_t (&v)[32], int cols) {
     if (p.use_red) {
@@ -439,6 +446,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 for (int c0 = 0; c0 < n_here; c0 += 64) {
                     tmem_ld_wait();
                     if (c0 + 32 < n_here) tmem_ld_32x32(t_row + c0 + 32, vb);
+                    if (p.out_f32) dequant_chunk(p, va);
                     if (p.c_mode == 1) tma_store_slab(p, staging, va, lane, q, warp == 2, tc.n0 + c0, m_cta);
                     else if (p.c_mode == 3) coalesced_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0);
                     else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging, va, lane, tc.n0 + c0, m_cta + q * 32);
@@ -446,6 +454,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     if (c0 + 32 < n_here) {
                         tmem_ld_wait();
                         if (c0 + 64 < n_here) tmem_ld_32x32(t_row + c0 + 64, va);
+                        if (p.out_f32) dequant_chunk(p, vb);
                         if (p.c_mode == 1) tma_store_slab(p, staging + 16384u, vb, lane, q, warp == 2, tc.n0 + c0 + 32, m_cta);
                         else if (p.c_mode == 3) coalesced_chunk(p, my_staging + 4096u, vb, lane, m_cta + q * 32, tc.n0 + c0 + 32);
                         else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + 4096u, vb, lane, tc.n0 + c0 + 32, m_cta + q * 32);
@@ -529,6 +538,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                         for (int e = 0; e < 4; ++e) v[4 * j + e] += x[e];
                     }
                 }
+                if (p.out_f32) dequant_chunk(p, v);
                 if (p.c_mode == 1) tma_store_slab(p, staging + (c & 1) * 16384u, v, lane, q, warp == 2, col0, m_cta);
                 else if (p.c_mode == 3) coalesced_chunk(p, my_staging + (c & 1) * 4096u, v, lane, m_cta + q * 32, col0);
                 else if (row < p.M) store_chunk(p, p.C + static_cast<long long>(row) * p.ldc + col0, v, min(32, p.N - col0));

@@ -37,6 +37,8 @@ struct alignas(64) DenseParams {
     int accumulate;          // epilogue adds the incoming C
     int use_red;             // epilogue reduces with red.global.add (split-K)
     int store_vec;           // 8, 4 or 1 int32 per store instruction
+    int out_f32;             // 1: the epilogue writes float32 scale * sum instead of the int32 sum
+    float out_scale;
     int c_mode;              // 0: row-per-thread stores (any alignment), 1: coalesced stores through
                              // shared memory, 2: TMA tile reduce-add (split-K); 1 and 2 need a 16-byte
                              // aligned C base and ldc % 4 == 0
@@ -64,6 +66,7 @@ struct SkinnyParams {
     int32_t* C; long long ldc;
     int M, N, K;
     int a_unsigned, accumulate;
+    int out_f32; float out_scale;   // fused dequantisation (see DenseParams)
 };
 cudaError_t launch_skinny(const SkinnyParams& p, cudaStream_t stream);
 bool skinny_supported(const SkinnyParams& p);
@@ -75,6 +78,7 @@ struct alignas(64) SkinnyRingParams {
     int32_t* C; long long ldc;
     int M, N, K;
     int a_unsigned, accumulate;
+    int out_f32; float out_scale;   // fused dequantisation (see DenseParams)
     int slots, tokens_in_smem;   // filled in by the launcher
     unsigned int* status;
     unsigned long long wait_budget_ns;

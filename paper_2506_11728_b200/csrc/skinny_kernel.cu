@@ -189,6 +189,7 @@ mip_skinny_kernel(const SkinnyParams p, int split) {
     if (tok < p.M && n0 + n < p.N) {
         int32_t* dst = p.C + static_cast<long long>(tok) * p.ldc + n0 + n;
         if (p.accumulate) sum = static_cast<int>(static_cast<uint32_t>(sum) + static_cast<uint32_t>(*dst));
+        if (p.out_f32) sum = __float_as_int(__int2float_rn(sum) * p.out_scale);   // fused dequantisation
         *dst = sum;
     }
 }

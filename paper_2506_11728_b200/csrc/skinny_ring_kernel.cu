@@ -236,6 +236,7 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
                 for (int w = 0; w < kRingConsumers; ++w) sum += red[w][n][tok];
                 int32_t* dst = p.C + static_cast<long long>(tok) * p.ldc + col;
                 if (p.accumulate) sum = static_cast<int>(static_cast<uint32_t>(sum) + static_cast<uint32_t>(*dst));
+                if (p.out_f32) sum = __float_as_int(__int2float_rn(sum) * p.out_scale);   // fused dequantisation
                 *dst = sum;
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");           // red[] may be overwritten

@@ -121,3 +121,16 @@ def test_implicit_im2col_cta_pair(mg, case):
         check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=41, accumulate=True)
     finally:
         mg.mipgemm_set_tuning()
+
+
+@pytest.mark.parametrize("layer", [0, 6, 14, 22])
+def test_resnet50_layers_batch128_sampled_images(mg, layer):
+    """Batch 128 (the largest configuration: the stem's GEMM has 1.6 M rows): full batch on the GPU,
+    three whole images recomputed by the oracle."""
+    _cnt, H, W, Cin, Cout, R, S, st, pd = inputs.RESNET50_CONVS[layer]
+    Nb = 128
+    X, Wt = conv_inputs(Nb, H, W, Cin, Cout, R, S, inputs.seed_for(3, layer) + 7)
+    got, _ = run_conv(mg, X, Wt, (st, st), (pd, pd), (1, 1))
+    for n in (0, 63, Nb - 1):
+        want = orc.conv(X[n:n + 1], Wt, stride=(st, st), pad=(pd, pd))
+        assert np.array_equal(got[n:n + 1], want), "image %d: %s" % (n, first_mismatch(got[n:n + 1], want))
