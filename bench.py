@@ -90,7 +90,7 @@ def build_square(torch, mg, sizes, keep_host):
     return probs
 
 
-def build_bert(torch, mg, tokens):
+def build_bert(torch, mg, tokens, dequant=False):
     probs = []
     for T in tokens:
         for (name, N, K) in inputs.BERT_GEMMS:
@@ -101,13 +101,17 @@ def build_bert(torch, mg, tokens):
             p = Problem("%s_T%d" % (name, T), "gemm", 2.0 * T * N * K, T * K + N * K + 4.0 * T * N)
             p.dims = (T, N, K)
             p.bufs = (dA, dB, dC)
-            p.calls = [lambda T=T, N=N, K=K, dA=dA, dB=dB, dC=dC:
-                       mg.mipgemm_s8s8s32(T, N, K, dA, K, dB, K, dC, N, 0)]
+            if dequant:
+                p.calls = [lambda T=T, N=N, K=K, dA=dA, dB=dB, dC=dC:
+                           mg.mipgemm_s8s8f32_dequant(T, N, K, dA, K, dB, K, dC, N, 1.25e-3)]
+            else:
+                p.calls = [lambda T=T, N=N, K=K, dA=dA, dB=dB, dC=dC:
+                           mg.mipgemm_s8s8s32(T, N, K, dA, K, dB, K, dC, N, 0)]
             probs.append(p)
     return probs
 
 
-def build_resnet(torch, mg, batch):
+def build_resnet(torch, mg, batch, dequant=False):
     probs = []
     for li, (cnt, H, W, Cin, Cout, R, S, st, pd) in enumerate(inputs.RESNET50_CONVS):
         Ho = (H + 2 * pd - (R - 1) - 1) // st + 1
@@ -122,8 +126,12 @@ def build_resnet(torch, mg, batch):
         p.dims = (M, Cout, K)
         p.count = cnt
         p.bufs = (dX, dW, dY)
-        p.calls = [lambda a=(batch, H, W, Cin, Cout, R, S, st, st, pd, pd, 1, 1), dX=dX, dW=dW, dY=dY:
-                   mg.mipgemm_conv_u8s8s32(*a, dX, dW, dY, 0)]
+        if dequant:
+            p.calls = [lambda a=(batch, H, W, Cin, Cout, R, S, st, st, pd, pd, 1, 1), dX=dX, dW=dW, dY=dY:
+                       mg.mipgemm_conv_u8s8f32_dequant(*a, dX, dW, dY, 7.5e-4)]
+        else:
+            p.calls = [lambda a=(batch, H, W, Cin, Cout, R, S, st, st, pd, pd, 1, 1), dX=dX, dW=dW, dY=dY:
+                       mg.mipgemm_conv_u8s8s32(*a, dX, dW, dY, 0)]
         probs.append(p)
     return probs
 
@@ -317,6 +325,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--detail", action="store_true", help="print per-problem timings to stderr")
     ap.add_argument("--eager", action="store_true", help="plain launches instead of CUDA-graph replay")
+    ap.add_argument("--dequant", action="store_true",
+                    help="bert/resnet: call the fused-dequantisation entry points (float32 = scale * sum)")
     ap.add_argument("--only", default="", help="keep only problems whose name contains this text (for profiling)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -348,11 +358,11 @@ def main():
         workload = "square s8*s8->s32 sweep M=N=K in %s, uniform int8, accumulate=0" % sizes
         unit, metric = "TOPS", "int8_gemm_tops"
     elif args.workload == "bert":
-        probs = build_bert(torch, mg, inputs.BERT_TOKENS)
+        probs = build_bert(torch, mg, inputs.BERT_TOKENS, args.dequant)
         workload = "BERT base/large encoder GEMMs s8*s8->s32, tokens %s" % inputs.BERT_TOKENS
         unit, metric = "TOPS", "int8_gemm_tops"
     elif args.workload == "resnet":
-        probs = build_resnet(torch, mg, args.batch)
+        probs = build_resnet(torch, mg, args.batch, args.dequant)
         workload = "ResNet-50 v1.5 convolutions u8*s8->s32 NHWC, batch %d, 53 layers" % args.batch
         unit, metric = "TOPS", "int8_conv_tops"
     else:
@@ -361,6 +371,8 @@ def main():
             inputs.SKINNY_M, inputs.SKINNY_WEIGHTS)
         unit, metric = "GB/s", "skinny_gemm_gbs"
 
+    if args.dequant and args.workload in ("bert", "resnet"):
+        workload += ", fused dequantisation to float32"
     if args.only:
         probs = [p for p in probs if args.only in p.name]
         workload += " [only: %s]" % args.only
