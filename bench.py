@@ -36,6 +36,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM traffic (bytes read + written) of the dominant kernel per launch, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that workload).
 NCU_TRAFFIC_BYTES = {
+    "paper_b1": None,
     "square": 1561e6,   # profiles/dense_kernel_square_sweep.md: (6.4 + 8.4 + 55.3 + 606.3 + 7128.4) MB / 5 launches
     "bert": None,
     "resnet": None,
@@ -132,6 +133,37 @@ def build_resnet(torch, mg, batch, dequant=False):
         else:
             p.calls = [lambda a=(batch, H, W, Cin, Cout, R, S, st, st, pd, pd, 1, 1), dX=dX, dW=dW, dY=dY:
                        mg.mipgemm_conv_u8s8s32(*a, dX, dW, dY, 0)]
+        probs.append(p)
+    return probs
+
+
+def build_paper_b1(torch, mg):
+    """The paper's own evaluation setting (Section 7.2): batch 1 -- all 53 ResNet-50 v1.5 convolutions
+    plus the final fully connected layer as a matrix-vector product (2048 -> 1000), and the six
+    weight GEMMs of one BERT-Large encoder block (Table 5) for one sentence of l = 512 tokens."""
+    probs = build_resnet(torch, mg, 1)
+    K, N = 2048, 1000
+    A = inputs.uniform_u8(K, inputs.seed_for(3, 99) + 1)
+    B = inputs.normal_s8(N * K, inputs.seed_for(3, 99) + 2, 32.0, -127, 127)
+    dA, dB = _dev_bytes(torch, A), _dev_bytes(torch, B)
+    dC = torch.empty(N, dtype=torch.int32, device="cuda")
+    p = Problem("fc_gemv_2048_1000", "gemm", 2.0 * N * K, N * K + K + 4.0 * N)
+    p.dims = (1, N, K)
+    p.count = 1
+    p.bufs = (dA, dB, dC)
+    p.calls = [lambda: mg.mipgemm_u8s8s32(1, N, K, dA, K, dB, K, dC, N, 0)]
+    probs.append(p)
+    T, d, f = 512, 1024, 4096
+    for (name, n, k, cnt) in [("M1-M3_qkv", d, d, 3), ("M9_attn_out", d, d, 1), ("F11_ffn1", f, d, 1), ("F13_ffn2", d, f, 1)]:
+        A = inputs.normal_s8(T * k, inputs.seed_for(4, n + k) + 1, 40.0)
+        B = inputs.normal_s8(n * k, inputs.seed_for(4, n + k) + 2, 20.0)
+        dA, dB = _dev_bytes(torch, A), _dev_bytes(torch, B)
+        dC = torch.empty(T * n, dtype=torch.int32, device="cuda")
+        p = Problem("bert_large_l512_%s" % name, "gemm", 2.0 * T * n * k, T * k + n * k + 4.0 * T * n)
+        p.dims = (T, n, k)
+        p.count = cnt
+        p.bufs = (dA, dB, dC)
+        p.calls = [lambda T=T, n=n, k=k, dA=dA, dB=dB, dC=dC: mg.mipgemm_s8s8s32(T, n, k, dA, k, dB, k, dC, n, 0)]
         probs.append(p)
     return probs
 
@@ -318,7 +350,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="square", choices=["square", "bert", "resnet", "skinny"])
+    ap.add_argument("--workload", default="square", choices=["square", "bert", "resnet", "skinny", "paper_b1"])
     ap.add_argument("--max-size", type=int, default=16384, help="largest member of the square sweep")
     ap.add_argument("--batch", type=int, default=32, help="resnet batch")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -365,6 +397,11 @@ def main():
         probs = build_resnet(torch, mg, args.batch, args.dequant)
         workload = "ResNet-50 v1.5 convolutions u8*s8->s32 NHWC, batch %d, 53 layers" % args.batch
         unit, metric = "TOPS", "int8_conv_tops"
+    elif args.workload == "paper_b1":
+        probs = build_paper_b1(torch, mg)
+        workload = ("the paper's batch-1 setting: ResNet-50 v1.5 (53 convs + FC matrix-vector product) and one "
+                    "BERT-Large encoder block, l = 512 (operands stay L2-resident at this size)")
+        unit, metric = "TOPS", "int8_b1_tops"
     else:
         probs = build_skinny(torch, mg)
         workload = "skinny decode GEMMs s8*s8->s32, M in %s, weights %s, rotated over >=512 MB" % (
@@ -383,7 +420,7 @@ def main():
     # rotation slots), grouped per problem so one event pair brackets each group
     groups = []
     for p in probs:
-        reps = getattr(p, "count", 1) if args.workload == "resnet" else len(p.calls)
+        reps = getattr(p, "count", 1) if args.workload in ("resnet", "paper_b1") else len(p.calls)
         groups.append((p, reps))
     launches_per_step = sum(r for (_p, r) in groups)
 
@@ -561,8 +598,10 @@ def main():
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "config": {"workload": workload,
-                   "l2": "operands + outputs of one step exceed the 126 MB L2 many times over; "
-                         "every buffer is evicted between two uses",
+                   "l2": ("operands stay L2-resident between steps (batch-1 problems are a few MB): a latency "
+                          "measurement, as in the paper's setting") if args.workload == "paper_b1" else
+                         ("operands + outputs of one step exceed the 126 MB L2 many times over; "
+                          "every buffer is evicted between two uses"),
                    "launches_per_step": launches_per_step,
                    "launch": "eager" if graph is None else "one CUDA graph replay per step"},
         "clocks": sampler.summary(),
