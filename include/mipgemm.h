@@ -78,7 +78,8 @@ typedef enum {
     MIPGEMM_PATH_REPACK = 0x100,  /* flag: an operand was re-pitched into scratch first      */
     MIPGEMM_PATH_SPLITK = 0x200,  /* flag: K was split and reduced with integer atomics      */
     MIPGEMM_PATH_IM2COL_TMA = 0x400,   /* flag: conv gathered by TMA im2col loads            */
-    MIPGEMM_PATH_IM2COL_EXPLICIT = 0x800 /* flag: conv materialised the augmented matrix     */
+    MIPGEMM_PATH_IM2COL_EXPLICIT = 0x800, /* flag: conv materialised the augmented matrix    */
+    MIPGEMM_PATH_BATCHED = 0x1000      /* flag: a whole strided batch ran as one launch       */
 } mipgemm_path_t;
 
 /*
@@ -126,6 +127,28 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
                          int pad_h, int pad_w, int dil_h, int dil_w,
                          const uint8_t *X, const int8_t *Wt, int32_t *Y,
                          int accumulate, void *stream);
+
+/*
+ * Strided batch of independent GEMMs:  C_b [+]= A_b * B_b,  b = 0 .. batch-1, with
+ * A_b = A + b*stride_a, B_b = B + b*stride_b, C_b = C + b*stride_c (strides in elements) and each
+ * member laid out exactly as in mipgemm_s8s8s32.  This is the shape of the per-head,
+ * per-sentence products of a transformer's attention (paper Table 5: M5, l x l x d/h, and M7,
+ * d/h x l x l), which the paper leaves in FP32; an int8 variant is offered here as the natural
+ * extension.  The C matrices must not overlap (stride_c >= (M-1)*ldc + N); stride_a / stride_b may
+ * be 0 to share an operand.  When all operands are 16-byte addressable (bases, pitches and batch
+ * strides) the batch runs as a single launch; otherwise the members are computed one after the
+ * other.  Same limits and return codes as the single GEMM.
+ */
+int mipgemm_batched_s8s8s32(int64_t batch, int64_t M, int64_t N, int64_t K,
+                            const int8_t *A, int64_t lda, int64_t stride_a,
+                            const int8_t *B, int64_t ldb, int64_t stride_b,
+                            int32_t *C, int64_t ldc, int64_t stride_c,
+                            int accumulate, void *stream);
+int mipgemm_batched_u8s8s32(int64_t batch, int64_t M, int64_t N, int64_t K,
+                            const uint8_t *A, int64_t lda, int64_t stride_a,
+                            const int8_t *B, int64_t ldb, int64_t stride_b,
+                            int32_t *C, int64_t ldc, int64_t stride_c,
+                            int accumulate, void *stream);
 
 /*
  * Fused dequantisation (paper Section 7.3: with A ~ s_A A^q and B ~ s_B B^q, the real-valued

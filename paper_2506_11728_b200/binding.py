@@ -29,12 +29,15 @@ STATIC_SCRATCH_BYTES = 8 << 20
 PATH_NONE, PATH_DENSE, PATH_DENSE_PAIR, PATH_SKINNY, PATH_TRIVIAL = range(5)
 PATH_MASK = 0xFF
 PATH_REPACK, PATH_SPLITK, PATH_IM2COL_TMA, PATH_IM2COL_EXPLICIT = 0x100, 0x200, 0x400, 0x800
+PATH_BATCHED = 0x1000
 
 #: every symbol include/mipgemm.h declares, with (restype, argtypes)
 SIGNATURES = {
     "mipgemm_s8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_u8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_conv_u8s8s32": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, _int, _vp]),
+    "mipgemm_batched_s8s8s32": (_int, [_i64] * 4 + [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _i64, _int, _vp]),
+    "mipgemm_batched_u8s8s32": (_int, [_i64] * 4 + [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _i64, _int, _vp]),
     "mipgemm_s8s8f32_dequant": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]),
     "mipgemm_u8s8f32_dequant": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]),
     "mipgemm_conv_u8s8f32_dequant": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, ctypes.c_float, _vp]),
@@ -107,6 +110,19 @@ def mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, p
     return _check(_lib.mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
                                             dil_h, dil_w, _ptr(X), _ptr(Wt), _ptr(Y),
                                             int(bool(accumulate)), _stream(stream)), check)
+
+
+def mipgemm_batched_s8s8s32(batch, M, N, K, A, lda, stride_a, B, ldb, stride_b, C, ldc, stride_c,
+                            accumulate=0, stream=None, check=True) -> int:
+    """C_b (+)= A_b * B_b for b < batch; member b of X starts stride_x elements after member b-1."""
+    return _check(_lib.mipgemm_batched_s8s8s32(batch, M, N, K, _ptr(A), lda, stride_a, _ptr(B), ldb, stride_b,
+                                               _ptr(C), ldc, stride_c, int(bool(accumulate)), _stream(stream)), check)
+
+
+def mipgemm_batched_u8s8s32(batch, M, N, K, A, lda, stride_a, B, ldb, stride_b, C, ldc, stride_c,
+                            accumulate=0, stream=None, check=True) -> int:
+    return _check(_lib.mipgemm_batched_u8s8s32(batch, M, N, K, _ptr(A), lda, stride_a, _ptr(B), ldb, stride_b,
+                                               _ptr(C), ldc, stride_c, int(bool(accumulate)), _stream(stream)), check)
 
 
 def mipgemm_s8s8f32_dequant(M, N, K, A, lda, B, ldb, C, ldc, scale, stream=None, check=True) -> int:

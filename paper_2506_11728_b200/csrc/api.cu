@@ -333,12 +333,17 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
     // shared memory, and split-K partial tiles are added into C by TMA tile reduce-adds.
     p.c_mode = 0;
     if (c_addr % 16 == 0 && ldc % 4 == 0 && !g_tuning_no_tma_store) {
+        // TMA tile stores clip at the tensor edge in 16-byte granules (measured: with N % 4 != 0 the
+        // columns N .. roundup(N,4)-1 were overwritten), so they are used only when N % 4 == 0; the
+        // coalesced path writes the ragged last columns one by one.
+        const bool tma_ok = N % 4 == 0;
         if (pl.split_k > 1 && !pl.cluster_split) {
-            p.c_mode = 2;
-            p.use_red = 0;
+            if (tma_ok) {
+                p.c_mode = 2;
+                p.use_red = 0;
+            }
         } else {
-            p.c_mode = accumulate ? 3 : 1;
-            if (const char* cm = std::getenv("MIPGEMM_CMODE")) p.c_mode = std::atoi(cm);
+            p.c_mode = (accumulate || !tma_ok) ? 3 : 1;
         }
     }
     p.out_f32 = tl_out_f32;
@@ -545,6 +550,108 @@ bool conv_tma_eligible(const ConvGeom& g, const void* X, const void* Wt) {
     if (g.W >= (1LL << 31) || g.H >= (1LL << 31) || g.Nb >= (1LL << 31)) return false;
     if (g.H * g.W * g.Cin >= (1LL << 40)) return false;
     return true;
+}
+
+// Strided batch: C_b [+]= A_b * B_b for b < batch.  When every operand of every batch member is
+// TMA-addressable the whole batch is one launch of the dense kernel (rank-3 tensor maps, the batch
+// index is the slowest tile coordinate); otherwise the members are served one by one.
+int batched_impl(bool a_unsigned, int64_t batch, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda,
+                 int64_t stride_a, const int8_t* B, int64_t ldb, int64_t stride_b, int32_t* C, int64_t ldc,
+                 int64_t stride_c, int accumulate, void* stream_v) {
+    tl_last_path = MIPGEMM_PATH_NONE;
+    if (batch < 0 || M < 0 || N < 0 || K < 0 || batch > 0x7FFFFFFFLL) return MIPGEMM_ERR_INVALID_ARG;
+    if (M > 0x7FFFFF00LL || N > 0x7FFFFF00LL) return MIPGEMM_ERR_INVALID_ARG;
+    if (lda < K || ldb < K || ldc < N || stride_a < 0 || stride_b < 0) return MIPGEMM_ERR_INVALID_ARG;
+    if (K > (a_unsigned ? 65793 : 131071)) return MIPGEMM_ERR_K_TOO_LARGE;
+    if (batch == 0 || M == 0 || N == 0) {
+        tl_last_path = MIPGEMM_PATH_TRIVIAL;
+        return MIPGEMM_OK;
+    }
+    if (batch > 1 && stride_c < (M - 1) * ldc + N) return MIPGEMM_ERR_INVALID_ARG;   // C matrices must not overlap
+    if (!C || reinterpret_cast<uintptr_t>(C) % 4 != 0) return MIPGEMM_ERR_INVALID_ARG;
+    if (K > 0 && (!A || !B)) return MIPGEMM_ERR_INVALID_ARG;
+    DeviceState* dev = nullptr;
+    int st = get_device(&dev);
+    if (st != MIPGEMM_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+
+    const long long tiles_m = (M + kBlockM - 1) / kBlockM;
+    const bool one_launch = batch > 1 && K > 0 && aligned16(A, lda) && aligned16(B, ldb) && stride_a % 16 == 0 &&
+                            stride_b % 16 == 0 && stride_a > 0 && stride_b > 0 && !tl_out_f32 &&
+                            tiles_m * ((N + 63) / 64) * batch < 0x7FFFFFFFLL;
+    if (!one_launch) {
+        int flags = 0;
+        for (int64_t b = 0; b < batch; ++b) {
+            st = gemm_impl(a_unsigned, M, N, K, static_cast<const char*>(A) + b * stride_a, lda, B + b * stride_b, ldb,
+                           C + b * stride_c, ldc, accumulate, stream_v, 0);
+            if (st != MIPGEMM_OK) return st;
+            flags |= tl_last_path;
+        }
+        tl_last_path = flags;
+        return MIPGEMM_OK;
+    }
+
+    const int block_k = K <= 64 ? 64 : 128;
+    Plan pl{};
+    pl.k_blocks = static_cast<int>((K + block_k - 1) / block_k);
+    double best = 1e30;
+    for (int bn = 64; bn <= 256; bn *= 2) {
+        if (g_tuning.block_n && bn != 64) continue;
+        const int bn_use = g_tuning.block_n ? g_tuning.block_n : bn;
+        const double us = plan_cost_us(0, bn_use, 1, tiles_m * batch * kBlockM, N, pl.k_blocks, block_k, dev);
+        if (us < best) { best = us; pl.block_n = bn_use; }
+    }
+    pl.pair = 0;
+    pl.cluster_split = 0;
+    pl.split_k = 1;
+    pl.kb_per_split = pl.k_blocks;
+    pl.tiles_m = static_cast<int>(tiles_m);
+    pl.tiles_n = static_cast<int>((N + pl.block_n - 1) / pl.block_n);
+    const int stage_bytes = kBlockM * block_k + pl.block_n * block_k;
+    int stages = (kSmemBudget - kCtrlBytes - kStagingBytes - 1024) / stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    pl.stages = stages;
+
+    DenseParams p;
+    std::memset(&p, 0, sizeof(p));
+    fill_common(p, pl, M, N, C, ldc, block_k, a_unsigned, accumulate, dev);
+    p.batch = static_cast<int>(batch);
+    p.stride_c = stride_c;
+    if (stride_c % 4 != 0 && p.c_mode != 0) {   // batch members of C would lose their 16-byte alignment
+        p.c_mode = 0;
+    }
+    auto encode3 = [&](CUtensorMap* map, const void* base, long long inner, long long rows, long long pitch,
+                       long long bstride, int box_inner, int box_rows, CUtensorMapDataType dt, int esize) -> int {
+        cuuint64_t dims[3] = {static_cast<cuuint64_t>(inner), static_cast<cuuint64_t>(rows),
+                              static_cast<cuuint64_t>(batch)};
+        cuuint64_t strides[2] = {static_cast<cuuint64_t>(pitch) * esize, static_cast<cuuint64_t>(bstride) * esize};
+        cuuint32_t box[3] = {static_cast<cuuint32_t>(box_inner), static_cast<cuuint32_t>(box_rows), 1};
+        cuuint32_t estr[3] = {1, 1, 1};
+        const CUtensorMapSwizzle sw = box_inner * esize == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+        CUresult r = g_encode_tiled(map, dt, 3, const_cast<void*>(base), dims, strides, box, estr,
+                                    CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            tl_last_cuda_error = 100000 + static_cast<int>(r);
+            return MIPGEMM_ERR_CUDA;
+        }
+        return MIPGEMM_OK;
+    };
+    if ((st = encode3(&p.tmap_a, A, K, M, lda, stride_a, block_k, kBlockM, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1)) != MIPGEMM_OK)
+        return st;
+    if ((st = encode3(&p.tmap_b, B, K, N, ldb, stride_b, block_k, pl.block_n, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1)) != MIPGEMM_OK)
+        return st;
+    if (p.c_mode == 1 &&
+        (st = encode3(&p.tmap_c, C, N, M, ldc, stride_c, 32, 128, CU_TENSOR_MAP_DATA_TYPE_INT32, 4)) != MIPGEMM_OK)
+        return st;
+    const long long units = tiles_m * pl.tiles_n * batch;
+    const int grid = static_cast<int>(units < dev->sm_count ? units : dev->sm_count);
+    const size_t smem = static_cast<size_t>(pl.stages) * stage_bytes + kStagingBytes + kCtrlBytes + 1024;
+    cudaError_t e = launch_dense(p, grid, smem, stream);
+    ++g_launches;
+    if (e != cudaSuccess) return cuda_fail(e);
+    tl_last_path = MIPGEMM_PATH_DENSE | MIPGEMM_PATH_BATCHED;
+    return MIPGEMM_OK;
 }
 
 // Host-buffer front end: stage operands, run the device entry point, copy C back.
@@ -759,6 +866,18 @@ int mipgemm_conv_u8s8f32_dequant(int64_t Nb, int64_t H, int64_t W, int64_t Cin, 
     OutputTransformScope scope(scale);
     return mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, X, Wt,
                                 reinterpret_cast<int32_t*>(Y), 0, stream);
+}
+
+int mipgemm_batched_s8s8s32(int64_t batch, int64_t M, int64_t N, int64_t K, const int8_t* A, int64_t lda,
+                            int64_t stride_a, const int8_t* B, int64_t ldb, int64_t stride_b, int32_t* C, int64_t ldc,
+                            int64_t stride_c, int accumulate, void* stream) {
+    return batched_impl(false, batch, M, N, K, A, lda, stride_a, B, ldb, stride_b, C, ldc, stride_c, accumulate, stream);
+}
+
+int mipgemm_batched_u8s8s32(int64_t batch, int64_t M, int64_t N, int64_t K, const uint8_t* A, int64_t lda,
+                            int64_t stride_a, const int8_t* B, int64_t ldb, int64_t stride_b, int32_t* C, int64_t ldc,
+                            int64_t stride_c, int accumulate, void* stream) {
+    return batched_impl(true, batch, M, N, K, A, lda, stride_a, B, ldb, stride_b, C, ldc, stride_c, accumulate, stream);
 }
 
 uint64_t mipgemm_launch_count(void) { return g_launches.load(); }

@@ -35,11 +35,16 @@ namespace mip {
 #endif
 
 struct TileCoord {
-    int m0, n0, kb_begin, kb_end;
+    int m0, n0, kb_begin, kb_end, batch;
 };
 
 __device__ __forceinline__ TileCoord decode_unit(const DenseParams& p, int unit, int rows_per_tile) {
     const int tiles_mn = p.tiles_m * p.tiles_n;
+    int batch = 0;
+    if (p.batch > 1) {                 // strided batch: the batch index is the slowest (no split-K)
+        batch = unit / tiles_mn;
+        unit -= batch * tiles_mn;
+    }
     // cluster split-K: the CTAs of a cluster (consecutive units) share one tile
     const int ks = p.cluster_split > 1 ? unit % p.cluster_split : unit / tiles_mn;
     const int t = p.cluster_split > 1 ? unit / p.cluster_split : unit - ks * tiles_mn;
@@ -57,6 +62,7 @@ __device__ __forceinline__ TileCoord decode_unit(const DenseParams& p, int unit,
     c.n0 = tn * p.block_n;
     c.kb_begin = ks * p.kb_per_split;
     c.kb_end = min(p.k_blocks, c.kb_begin + p.kb_per_split);
+    c.batch = batch;
     return c;
 }
 
@@ -129,7 +135,7 @@ __device__ __forceinline__ void tma_reduce_chunk(const DenseParams& p, uint32_t 
 // meet at a named barrier, and one thread issues the store, which clips at the edges of C.
 // `buf` alternates between two buffers; `issuer` is true in exactly one warp.
 __device__ __forceinline__ void tma_store_slab(const DenseParams& p, uint32_t buf, const uint32_t (&v)[32],
-                                               int lane, int q, bool issuer, int x, int y) {
+                                               int lane, int q, bool issuer, int x, int y, int z = 0) {
     if (issuer && elect_one()) tma_store_wait_read<1>();
     asm volatile("bar.sync 1, 128;" ::: "memory");      // the buffer is free for all four warps
     const int r = q * 32 + lane;
@@ -139,7 +145,8 @@ __device__ __forceinline__ void tma_store_slab(const DenseParams& p, uint32_t bu
     fence_proxy_async_smem();
     asm volatile("bar.sync 1, 128;" ::: "memory");      // all 128 rows are in place
     if (issuer && elect_one()) {
-        tma_store_2d(&p.tmap_c, buf, x, y);
+        if (p.batch > 1) tma_store_3d(&p.tmap_c, buf, x, y, z);
+        else tma_store_2d(&p.tmap_c, buf, x, y);
         tma_store_commit();
     }
 }
@@ -150,7 +157,7 @@ __device__ __forceinline__ void tma_store_slab(const DenseParams& p, uint32_t bu
 // incoming C is read with the same access pattern and added.  Needs a 16-byte aligned C
 // base and ldc % 4 == 0.  (row0, col0) is the chunk's origin in C.
 __device__ __forceinline__ void coalesced_chunk(const DenseParams& p, uint32_t buf, const uint32_t (&v)[32],
-                                                int lane, int row0, int col0) {
+                                                int lane, int row0, int col0, long long c_off = 0) {
     __syncwarp();   // the previous chunk's reads of `buf` are done
     const uint32_t mine = buf + static_cast<uint32_t>(lane) * 128u;
 #pragma unroll
@@ -169,7 +176,7 @@ __device__ __forceinline__ void coalesced_chunk(const DenseParams& p, uint32_t b
             : "r"(buf + static_cast<uint32_t>(r) * 128u + (static_cast<uint32_t>(piece ^ (r & 7)) << 4))
             : "memory");
     }
-    int32_t* dst0 = p.C + static_cast<long long>(row0 + (lane >> 3)) * p.ldc + col;
+    int32_t* dst0 = p.C + c_off + static_cast<long long>(row0 + (lane >> 3)) * p.ldc + col;
     const long long step = 4 * p.ldc;
     if (p.accumulate && cols_left >= 4) {
         uint32_t c[8][4];
@@ -276,7 +283,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
     const uint32_t tmem_base = *tmem_slot;
     if (threadIdx.x == 0) MIP_STAMP(1);
 
-    const int total_units = p.tiles_m * p.tiles_n * p.split_k;
+    const int total_units = p.tiles_m * p.tiles_n * p.split_k * (p.batch > 1 ? p.batch : 1);
     const uint64_t budget = p.wait_budget_ns;
 
     if (warp == 0) {
@@ -326,11 +333,15 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                                                static_cast<uint16_t>(fr * p.dil_h));
                     } else if (kPair) {
                         tma_load_2d_pair(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta);
+                    } else if (p.batch > 1) {
+                        tma_load_3d(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta, tc.batch);
                     } else {
                         tma_load_2d(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta);
                     }
                     if (kPair)
                         tma_load_2d_pair(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta);
+                    else if (p.batch > 1)
+                        tma_load_3d(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta, tc.batch);
                     else
                         tma_load_2d(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta);
                 }
@@ -436,7 +447,8 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             if (p.cluster_split > 1) {
                 // the accumulator stays in tensor memory; the cluster reduces it below
             } else if (p.c_mode == 1 || m_cta + q * 32 < p.M) {   // (slab stores need all four warps)
-                int32_t* crow = p.C + static_cast<long long>(row) * p.ldc + tc.n0;
+                const long long c_off = static_cast<long long>(tc.batch) * p.stride_c;
+                int32_t* crow = p.C + c_off + static_cast<long long>(row) * p.ldc + tc.n0;
                 const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.block_n;
                 const uint32_t my_staging = staging + static_cast<uint32_t>(q) * 8192u;
                 // two register buffers: the TMEM load of the next chunk is in flight while the
@@ -447,16 +459,16 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     tmem_ld_wait();
                     if (c0 + 32 < n_here) tmem_ld_32x32(t_row + c0 + 32, vb);
                     if (p.out_f32) dequant_chunk(p, va);
-                    if (p.c_mode == 1) tma_store_slab(p, staging, va, lane, q, warp == 2, tc.n0 + c0, m_cta);
-                    else if (p.c_mode == 3) coalesced_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0);
+                    if (p.c_mode == 1) tma_store_slab(p, staging, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
+                    else if (p.c_mode == 3) coalesced_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
                     else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging, va, lane, tc.n0 + c0, m_cta + q * 32);
                     else if (row < p.M) store_chunk(p, crow + c0, va, min(32, n_here - c0));
                     if (c0 + 32 < n_here) {
                         tmem_ld_wait();
                         if (c0 + 64 < n_here) tmem_ld_32x32(t_row + c0 + 64, va);
                         if (p.out_f32) dequant_chunk(p, vb);
-                        if (p.c_mode == 1) tma_store_slab(p, staging + 16384u, vb, lane, q, warp == 2, tc.n0 + c0 + 32, m_cta);
-                        else if (p.c_mode == 3) coalesced_chunk(p, my_staging + 4096u, vb, lane, m_cta + q * 32, tc.n0 + c0 + 32);
+                        if (p.c_mode == 1) tma_store_slab(p, staging + 16384u, vb, lane, q, warp == 2, tc.n0 + c0 + 32, m_cta, tc.batch);
+                        else if (p.c_mode == 3) coalesced_chunk(p, my_staging + 4096u, vb, lane, m_cta + q * 32, tc.n0 + c0 + 32, c_off);
                         else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + 4096u, vb, lane, tc.n0 + c0 + 32, m_cta + q * 32);
                         else if (row < p.M) store_chunk(p, crow + c0 + 32, vb, min(32, n_here - c0 - 32));
                     }

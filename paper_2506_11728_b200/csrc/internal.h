@@ -32,6 +32,8 @@ struct alignas(64) DenseParams {
     int stages;
     int tiles_m, tiles_n;
     int split_k, kb_per_split;
+    int batch;               // > 1: strided batch; the tensor maps are rank 3 (z = batch index)
+    long long stride_c;      // elements between consecutive C matrices of a batch
     int cluster_split;       // > 1: the split_k CTAs sharing a tile form a cluster and reduce through DSMEM
     int group_n;             // n-tiles per rasterisation group
     int accumulate;          // epilogue adds the incoming C

@@ -63,14 +63,6 @@ __device__ __forceinline__ uint4 ldg_tokens(const uint8_t* p, bool valid) {
     return r;
 }
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* m, uint32_t bar, int32_t x,
-                                            int32_t y, int32_t z) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
-}
-
 struct TokenRegs {
     uint4 x0l, x0h, x1l, x1h;
 };

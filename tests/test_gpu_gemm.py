@@ -247,3 +247,20 @@ def test_cta_pair_with_unaligned_c_and_repack(mg):
         check_case(mg, "u8", 515, 259, 400, ldc=261, seed=461)
     finally:
         mg.mipgemm_set_tuning()
+
+
+def test_padding_columns_survive_when_n_is_not_a_multiple_of_four(mg):
+    """A 16-byte aligned C with N % 4 != 0: tile stores must not spill into the padding columns."""
+    for (M, N, K, ldc) in [(300, 70, 400, 72), (257, 1001, 272, 1004), (129, 34, 144, 40)]:
+        check_case(mg, "s8", M, N, K, ldc=ldc, seed=500 + N)
+        check_case(mg, "u8", M, N, K, ldc=ldc, seed=510 + N, accumulate=True)
+    mg.mipgemm_set_tuning(split_k=3)
+    try:
+        check_case(mg, "s8", 200, 70, 1296, ldc=72, seed=520)
+    finally:
+        mg.mipgemm_set_tuning()
+    mg.mipgemm_set_tuning(force_path=mg.PATH_DENSE_PAIR)
+    try:
+        check_case(mg, "s8", 600, 1001, 400, ldc=1004, seed=530)
+    finally:
+        mg.mipgemm_set_tuning()
