@@ -36,6 +36,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM traffic (bytes read + written) of the dominant kernel per launch, from the ncu
 # captures summarised under profiles/ (None until a capture exists for that workload).
 NCU_TRAFFIC_BYTES = {
+    "attention": None,
     "paper_b1": None,
     "square": 1561e6,   # profiles/dense_kernel_square_sweep.md: (6.4 + 8.4 + 55.3 + 606.3 + 7128.4) MB / 5 launches
     "bert": None,
@@ -164,6 +165,26 @@ def build_paper_b1(torch, mg):
         p.count = cnt
         p.bufs = (dA, dB, dC)
         p.calls = [lambda T=T, n=n, k=k, dA=dA, dB=dB, dC=dC: mg.mipgemm_s8s8s32(T, n, k, dA, k, dB, k, dC, n, 0)]
+        probs.append(p)
+    return probs
+
+
+def build_attention(torch, mg, sentences=8, heads=16, l=512, dh=64):
+    """The activation-by-activation products of BERT-Large's attention (paper Table 5): M5, l x l x d/h,
+    and M7, d/h x l x l, one per head and sentence, as strided int8 batches."""
+    batch = sentences * heads
+    probs = []
+    for (name, M, N, K) in [("M5_scores", l, l, dh), ("M7_context", l, dh, l)]:
+        A = inputs.normal_s8(batch * M * K, inputs.seed_for(4, 900 + K) + 1, 40.0)
+        B = inputs.normal_s8(batch * N * K, inputs.seed_for(4, 900 + K) + 2, 40.0)
+        dA, dB = _dev_bytes(torch, A), _dev_bytes(torch, B)
+        dC = torch.empty(batch * M * N, dtype=torch.int32, device="cuda")
+        p = Problem("attention_%s_x%d" % (name, batch), "gemm", 2.0 * batch * M * N * K,
+                    batch * (M * K + N * K + 4.0 * M * N))
+        p.dims = (M, N, K)
+        p.bufs = (dA, dB, dC)
+        p.calls = [lambda M=M, N=N, K=K, dA=dA, dB=dB, dC=dC:
+                   mg.mipgemm_batched_s8s8s32(batch, M, N, K, dA, K, M * K, dB, K, N * K, dC, N, M * N, 0)]
         probs.append(p)
     return probs
 
@@ -350,7 +371,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="square", choices=["square", "bert", "resnet", "skinny", "paper_b1"])
+    ap.add_argument("--workload", default="square", choices=["square", "bert", "resnet", "skinny", "paper_b1", "attention"])
     ap.add_argument("--max-size", type=int, default=16384, help="largest member of the square sweep")
     ap.add_argument("--batch", type=int, default=32, help="resnet batch")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -397,6 +418,10 @@ def main():
         probs = build_resnet(torch, mg, args.batch, args.dequant)
         workload = "ResNet-50 v1.5 convolutions u8*s8->s32 NHWC, batch %d, 53 layers" % args.batch
         unit, metric = "TOPS", "int8_conv_tops"
+    elif args.workload == "attention":
+        probs = build_attention(torch, mg)
+        workload = "BERT-Large attention products M5 (512x512x64) and M7 (512x64x512) as strided int8 batches of 128"
+        unit, metric = "TOPS", "int8_batched_tops"
     elif args.workload == "paper_b1":
         probs = build_paper_b1(torch, mg)
         workload = ("the paper's batch-1 setting: ResNet-50 v1.5 (53 convs + FC matrix-vector product) and one "
