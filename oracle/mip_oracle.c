@@ -14,7 +14,8 @@
  *   R(i,j) = (accumulate ? C_in(i,j) : 0) + sum_{k<K} a(i,k) * b(k,j)
  *
  * evaluated in 64-bit integers, a(i,k) sign-extended (int8) or zero-extended
- * (uint8), b(k,j) sign-extended, and then required to fit int32.  A cell whose
+ * (uint8), b(k,j) sign-extended (or, through mip_oracle_gemm_ex, zero-extended),
+ * and then required to fit int32.  A cell whose
  * exact value does not fit is counted as an overflow cell (the result there is
  * the low 32 bits, and callers treat the configuration as invalid).
  *
@@ -51,10 +52,10 @@ static inline int64_t widen_a(const void *A, int64_t idx, int a_unsigned)
  * Returns the number of overflow cells (0 = every cell fits int32), or -1 on
  * invalid arguments.
  */
-int64_t mip_oracle_gemm(int a_unsigned, int64_t M, int64_t N, int64_t K,
-                        const void *A, int64_t lda,
-                        const int8_t *B, int64_t ldb,
-                        int32_t *C, int64_t ldc, int accumulate)
+int64_t mip_oracle_gemm_ex(int a_unsigned, int b_unsigned, int64_t M, int64_t N, int64_t K,
+                           const void *A, int64_t lda,
+                           const void *B, int64_t ldb,
+                           int32_t *C, int64_t ldc, int accumulate)
 {
     if (M < 0 || N < 0 || K < 0)
         return -1;
@@ -72,7 +73,7 @@ int64_t mip_oracle_gemm(int a_unsigned, int64_t M, int64_t N, int64_t K,
             int64_t S = 0;
             for (int64_t k = 0; k < K; ++k) {
                 int64_t a = widen_a(A, i * lda + k, a_unsigned);
-                int64_t b = (int64_t)B[j * ldb + k];
+                int64_t b = widen_a(B, j * ldb + k, b_unsigned);
                 S += a * b;
             }
             int64_t R = (accumulate ? (int64_t)C[i * ldc + j] : 0) + S;
@@ -82,6 +83,15 @@ int64_t mip_oracle_gemm(int a_unsigned, int64_t M, int64_t N, int64_t K,
         }
     }
     return overflow_cells;
+}
+
+/* The common case: B signed. */
+int64_t mip_oracle_gemm(int a_unsigned, int64_t M, int64_t N, int64_t K,
+                        const void *A, int64_t lda,
+                        const int8_t *B, int64_t ldb,
+                        int32_t *C, int64_t ldc, int accumulate)
+{
+    return mip_oracle_gemm_ex(a_unsigned, 0, M, N, K, A, lda, B, ldb, C, ldc, accumulate);
 }
 
 /*

@@ -45,6 +45,8 @@ def _load():
         i64, vp, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
         lib.mip_oracle_gemm.restype = i64
         lib.mip_oracle_gemm.argtypes = [ci, i64, i64, i64, vp, i64, vp, i64, vp, i64, ci]
+        lib.mip_oracle_gemm_ex.restype = i64
+        lib.mip_oracle_gemm_ex.argtypes = [ci, ci, i64, i64, i64, vp, i64, vp, i64, vp, i64, ci]
         lib.mip_oracle_conv.restype = i64
         lib.mip_oracle_conv.argtypes = [i64] * 13 + [vp, vp, vp, ci]
         lib.mip_oracle_dequant.restype = None
@@ -74,7 +76,7 @@ def gemm(A: np.ndarray, B: np.ndarray, M: int, N: int, K: int, *, lda: int | Non
     """C = [C +] A * B, exact.
 
     ``A``: flat or 2-D C-contiguous buffer of int8 (signed mode) or uint8
-    (unsigned mode), row-major M x K with pitch ``lda``.  ``B``: int8 buffer,
+    (unsigned mode), row-major M x K with pitch ``lda``.  ``B``: int8 (or uint8) buffer,
     column-major K x N, i.e. N runs of K bytes with pitch ``ldb``.  ``C``:
     int32 buffer with pitch ``ldc`` (allocated, zero-filled, when omitted); it is
     updated in place and returned.  Raises :class:`OracleOverflow` if any exact
@@ -86,8 +88,12 @@ def gemm(A: np.ndarray, B: np.ndarray, M: int, N: int, K: int, *, lda: int | Non
         a_unsigned = 1
     else:
         raise TypeError("A must be int8 or uint8")
-    if B.dtype != np.int8:
-        raise TypeError("B must be int8")
+    if B.dtype == np.int8:
+        b_unsigned = 0
+    elif B.dtype == np.uint8:
+        b_unsigned = 1
+    else:
+        raise TypeError("B must be int8 or uint8")
     lda = K if lda is None else lda
     ldb = K if ldb is None else ldb
     ldc = N if ldc is None else ldc
@@ -103,8 +109,8 @@ def gemm(A: np.ndarray, B: np.ndarray, M: int, N: int, K: int, *, lda: int | Non
             raise ValueError("A or B buffer too small for the stated pitch")
         if C.size < (M - 1) * ldc + N:
             raise ValueError("C buffer too small for the stated pitch")
-    rc = _load().mip_oracle_gemm(a_unsigned, M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
-                                 1 if accumulate else 0)
+    rc = _load().mip_oracle_gemm_ex(a_unsigned, b_unsigned, M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                    1 if accumulate else 0)
     if rc < 0:
         raise ValueError("mip_oracle_gemm rejected its arguments")
     if rc > 0 and not allow_overflow:

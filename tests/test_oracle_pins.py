@@ -313,3 +313,32 @@ def test_dequant_closed_forms():
         assert Fraction(g) == Fraction(c) * Fraction(s)
     two_d = orc.dequant(Cq[:6].reshape(2, 3), 3.0)
     assert two_d.shape == (2, 3) and two_d[1, 2] == 3.0 * 16777217
+
+
+# ---------------------------------------------------------------------------
+# Unsigned B (all four signedness pairs): extremes, brute force, NumPy.
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("a_dt,b_dt,a_val,b_val", [
+    (np.uint8, np.uint8, 255, 255), (np.int8, np.uint8, -128, 255), (np.int8, np.uint8, 127, 255),
+    (np.uint8, np.uint8, 1, 200)])
+def test_unsigned_b_extremes(a_dt, b_dt, a_val, b_val):
+    M, N, K = 2, 3, 500
+    A = np.full(M * K, a_val, dtype=a_dt)
+    B = np.full(N * K, b_val, dtype=b_dt)
+    assert (orc.gemm(A, B, M, N, K) == a_val * b_val * K).all()      # 200 and 255 really are 200 and 255
+
+
+def test_unsigned_b_matches_numpy_and_brute_force():
+    rng = np.random.default_rng(77)
+    for a_dt in (np.int8, np.uint8):
+        M, N, K = 23, 17, 45
+        A = rng.integers(0, 256, size=M * K).astype(np.uint8).view(a_dt)
+        B = rng.integers(0, 256, size=N * K).astype(np.uint8)
+        want = A.reshape(M, K).astype(np.int64) @ B.reshape(N, K).astype(np.int64).T
+        got = orc.gemm(A, B, M, N, K).reshape(M, N)
+        assert (got.astype(np.int64) == want).all()
+    # u8 x u8 range guard: 255 * 255 * 33025 = 2147450625 fits, 33026 does not
+    Au = np.full(33026, 255, dtype=np.uint8)
+    assert int(orc.gemm(Au[:33025], Au[:33025], 1, 1, 33025)[0]) == 255 * 255 * 33025
+    with pytest.raises(orc.OracleOverflow):
+        orc.gemm(Au, Au, 1, 1, 33026)
