@@ -5,7 +5,7 @@ A *step* is one pass of the hot path over one batch of synthetic input: every GE
 convolution) of the chosen workload, launched back to back on one stream through the C
 ABI.  The default workload is the square s8*s8->s32 sweep M=N=K in {1024 .. 16384}.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload square|bert|resnet|skinny]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload square|bert|resnet|skinny|paper_b1|attention|layouts]
     python bench.py --impl reference ...      # the CPU oracle, timed on the host cores
 
 Under torchrun (N > 1) every rank runs the same per-GPU workload on its own device
@@ -89,6 +89,25 @@ def build_square(torch, mg, sizes, keep_host):
         if keep_host:
             p.host = (A, B)
         probs.append(p)
+    return probs
+
+
+def build_layouts(torch, mg, n=8192):
+    """The same square product under every storage-order combination of A, B and C."""
+    A = inputs.uniform_s8(n * n, inputs.seed_for(8, n) + 1)
+    B = inputs.uniform_s8(n * n, inputs.seed_for(8, n) + 2)
+    dA, dB = _dev_bytes(torch, A), _dev_bytes(torch, B)
+    dC = torch.empty(n * n, dtype=torch.int32, device="cuda")
+    probs = []
+    for ao in (0, 1):
+        for bo in (0, 1):
+            for cc in (0, 1):
+                p = Problem("A%s_B%s_C%s_%d" % ("km"[ao], "kn"[bo], "rc"[cc], n), "gemm", 2.0 * n ** 3, 6.0 * n * n)
+                p.dims = (n, n, n)
+                p.bufs = (dA, dB, dC)
+                p.calls = [lambda ao=ao, bo=bo, cc=cc: mg.mipgemm_gemm_ex(0, 0, ao, bo, cc, n, n, n, dA, n, dB, n,
+                                                                          dC, n, 0)]
+                probs.append(p)
     return probs
 
 
@@ -371,7 +390,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="square", choices=["square", "bert", "resnet", "skinny", "paper_b1", "attention"])
+    ap.add_argument("--workload", default="square", choices=["square", "bert", "resnet", "skinny", "paper_b1", "attention",
+                                                                "layouts"])
     ap.add_argument("--max-size", type=int, default=16384, help="largest member of the square sweep")
     ap.add_argument("--batch", type=int, default=32, help="resnet batch")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -422,6 +442,11 @@ def main():
         probs = build_attention(torch, mg)
         workload = "BERT-Large attention products M5 (512x512x64) and M7 (512x64x512) as strided int8 batches of 128"
         unit, metric = "TOPS", "int8_batched_tops"
+    elif args.workload == "layouts":
+        probs = build_layouts(torch, mg)
+        workload = ("8192^3 s8*s8->s32 under the eight storage-order combinations (A K-/M-contiguous, "
+                    "B K-/N-contiguous, C row-/column-major)")
+        unit, metric = "TOPS", "int8_gemm_tops"
     elif args.workload == "paper_b1":
         probs = build_paper_b1(torch, mg)
         workload = ("the paper's batch-1 setting: ResNet-50 v1.5 (53 convs + FC matrix-vector product) and one "
@@ -549,7 +574,7 @@ def main():
     # average launch duration is the region's elapsed time over its launches
     kernel_ms = elapsed_ms
     n_launch = launches_per_step * args.steps
-    if unit == "TOPS" and args.workload in ("square", "bert"):
+    if unit == "TOPS" and args.workload in ("square", "bert", "layouts"):
         int8_burst = peaks["bf16_tflops"] * (NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS)
         int8_sust = peaks["bf16_tflops_sustained"] * (NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS)
         achieved = args.steps * step_ops / (kernel_ms * 1e-3) / 1e12
@@ -557,7 +582,7 @@ def main():
                     "unit": "TFLOP/s", "frac": achieved / int8_burst,
                     "peak_source": "%s bf16 cuBLAS burst x2 (nominal int8:bf16 ratio)" % peaks["_source"],
                     "frac_of_sustained": achieved / int8_sust, "frac_of_nominal_4500": achieved / NOMINAL_INT8_TOPS,
-                    "traffic": NCU_TRAFFIC_BYTES[args.workload]}
+                    "traffic": NCU_TRAFFIC_BYTES.get(args.workload)}
     else:
         achieved = args.steps * step_bytes / (kernel_ms * 1e-3) / 1e9
         kname = "mip_skinny_kernel" if args.workload == "skinny" else "mip_dense_kernel"

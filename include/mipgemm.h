@@ -129,6 +129,28 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
                          int accumulate, void *stream);
 
 /*
+ * General form (paper Section 3, last paragraph: a general GEMM supports transposed inputs and
+ * both storage orders for all three operands; the effects on A and B are absorbed below the
+ * micro-kernel and a column-major C is handled by swapping the roles of A and B).
+ *
+ *   a_unsigned, b_unsigned : 0 = int8 (sign-extended), 1 = uint8 (zero-extended), per operand
+ *   a_order : MIPGEMM_K_CONTIGUOUS  a(i,k) = A[i*lda + k] (row-major,    lda >= K)
+ *             MIPGEMM_MN_CONTIGUOUS a(i,k) = A[k*lda + i] (column-major, lda >= M)
+ *   b_order : MIPGEMM_K_CONTIGUOUS  b(k,j) = B[j*ldb + k] (column-major, ldb >= K)
+ *             MIPGEMM_MN_CONTIGUOUS b(k,j) = B[k*ldb + j] (row-major,    ldb >= N)
+ *   c_col_major : 0  c(i,j) = C[i*ldc + j] (ldc >= N);  1  c(i,j) = C[j*ldc + i] (ldc >= M)
+ *
+ * K limits for a guaranteed exact result: 131071 (s8*s8), 65793 (one operand unsigned), 33025
+ * (u8*u8).  Operands whose base or pitch is not 16-byte aligned are re-pitched (transposed, when
+ * M/N-contiguous) into scratch memory first.  Everything else as for mipgemm_s8s8s32.
+ */
+typedef enum { MIPGEMM_K_CONTIGUOUS = 0, MIPGEMM_MN_CONTIGUOUS = 1 } mipgemm_order_t;
+int mipgemm_gemm_ex(int a_unsigned, int b_unsigned, int a_order, int b_order, int c_col_major,
+                    int64_t M, int64_t N, int64_t K,
+                    const void *A, int64_t lda, const void *B, int64_t ldb,
+                    int32_t *C, int64_t ldc, int accumulate, void *stream);
+
+/*
  * Strided batch of independent GEMMs:  C_b [+]= A_b * B_b,  b = 0 .. batch-1, with
  * A_b = A + b*stride_a, B_b = B + b*stride_b, C_b = C + b*stride_c (strides in elements) and each
  * member laid out exactly as in mipgemm_s8s8s32.  This is the shape of the per-head,

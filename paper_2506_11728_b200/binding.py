@@ -36,6 +36,7 @@ SIGNATURES = {
     "mipgemm_s8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_u8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_conv_u8s8s32": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, _int, _vp]),
+    "mipgemm_gemm_ex": (_int, [_int] * 5 + [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_batched_s8s8s32": (_int, [_i64] * 4 + [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _i64, _int, _vp]),
     "mipgemm_batched_u8s8s32": (_int, [_i64] * 4 + [_vp, _i64, _i64, _vp, _i64, _i64, _vp, _i64, _i64, _int, _vp]),
     "mipgemm_s8s8f32_dequant": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]),
@@ -110,6 +111,17 @@ def mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, p
     return _check(_lib.mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
                                             dil_h, dil_w, _ptr(X), _ptr(Wt), _ptr(Y),
                                             int(bool(accumulate)), _stream(stream)), check)
+
+
+K_CONTIGUOUS, MN_CONTIGUOUS = 0, 1
+
+
+def mipgemm_gemm_ex(a_unsigned, b_unsigned, a_order, b_order, c_col_major, M, N, K, A, lda, B, ldb, C, ldc,
+                    accumulate=0, stream=None, check=True) -> int:
+    """General GEMM: any signedness pair, either storage order for A and B, row- or column-major C."""
+    return _check(_lib.mipgemm_gemm_ex(int(a_unsigned), int(b_unsigned), int(a_order), int(b_order),
+                                       int(c_col_major), M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                       int(bool(accumulate)), _stream(stream)), check)
 
 
 def mipgemm_batched_s8s8s32(batch, M, N, K, A, lda, stride_a, B, ldb, stride_b, C, ldc, stride_c,

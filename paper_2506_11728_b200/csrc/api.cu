@@ -230,7 +230,8 @@ double plan_cost_us(int pair, int bn, int split, long long M, long long N, int k
     return 3.7 + (pair ? 1.0 : 0.0) + clk / 1900.0;   // pairs: cluster launch, two cluster barriers
 }
 
-Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceState* dev) {
+Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceState* dev, bool allow_pair = true,
+               int min_bn = 64) {
     const int sm_count = dev->sm_count;
     Plan pl{};
     pl.k_blocks = static_cast<int>((K + block_k - 1) / block_k);
@@ -238,19 +239,22 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
     // Candidates: one CTA per tile or CTA pairs, bn in {64, 128, 256}, optionally a cluster
     // split-K of 2/4/8 when the tiles alone would leave most SMs idle.  Experiment overrides
     // (mipgemm_set_tuning) restrict the candidate set.
-    int best_pair = 0, best_bn = g_tuning.block_n ? g_tuning.block_n : 128, best_split = 1;
+    int best_pair = 0, best_bn = 128, best_split = 1;
     double best = 1e30;
     // (an explicit split reduces int32 tiles in global memory, which a float output cannot share)
     const bool explicit_split = g_tuning.split_k != 0 && !tl_out_f32;
+    // (N-contiguous B tiles come in 128-column blocks: only 128 and 256 can be forced there)
+    const int forced_bn = (g_tuning.block_n && (min_bn <= 64 || g_tuning.block_n % 128 == 0)) ? g_tuning.block_n : 0;
     for (int pair = 0; pair <= 1; ++pair) {
-        if (pair && dev->pair_clusters <= 0) continue;
+        if (pair && (dev->pair_clusters <= 0 || !allow_pair)) continue;
         if (g_tuning.force_path == MIPGEMM_PATH_DENSE_PAIR && !pair && dev->pair_clusters > 0) continue;
         if (g_tuning.force_path == MIPGEMM_PATH_DENSE && pair) continue;
         for (int bn = 64; bn <= 256; bn *= 2) {
             int bn_use = bn;
-            if (g_tuning.block_n) {
-                if (bn != 64) continue;                       // a single candidate: the forced width
-                bn_use = g_tuning.block_n;
+            if (bn < min_bn) continue;
+            if (forced_bn) {
+                if (bn != 256) continue;                      // a single candidate: the forced width
+                bn_use = forced_bn;
                 if (pair && bn_use % 64 != 0) bn_use = (bn_use + 63) / 64 * 64;
             }
             const long long rows = pair ? 2 * kBlockM : kBlockM;
@@ -550,6 +554,95 @@ bool conv_tma_eligible(const ConvGeom& g, const void* X, const void* Wt) {
     if (g.W >= (1LL << 31) || g.H >= (1LL << 31) || g.Nb >= (1LL << 31)) return false;
     if (g.H * g.W * g.Cin >= (1LL << 40)) return false;
     return true;
+}
+
+// General form: any signedness pair, either storage order for A and B, row- or column-major C
+// (paper Section 3: transposition and storage order are absorbed below the micro-kernel; a
+// column-major C by swapping the roles of A and B).  M- / N-contiguous operands are read by the
+// tensor cores as they are (MN-major shared-memory descriptors); only operands TMA cannot
+// address are first transposed into K-contiguous scratch.
+int gemm_ex_impl(int a_unsigned, int b_unsigned, int a_order, int b_order, int c_col_major, int64_t M, int64_t N,
+                 int64_t K, const void* A, int64_t lda, const void* B, int64_t ldb, int32_t* C, int64_t ldc,
+                 int accumulate, void* stream_v) {
+    tl_last_path = MIPGEMM_PATH_NONE;
+    if ((a_order | b_order | c_col_major | a_unsigned | b_unsigned) & ~1) return MIPGEMM_ERR_INVALID_ARG;
+    if (c_col_major)   // C^T = B^T A^T: the same problem with the operands' roles exchanged
+        return gemm_ex_impl(b_unsigned, a_unsigned, b_order, a_order, 0, N, M, K, B, ldb, A, lda, C, ldc, accumulate,
+                            stream_v);
+    if (M < 0 || N < 0 || K < 0 || M > 0x7FFFFF00LL || N > 0x7FFFFF00LL) return MIPGEMM_ERR_INVALID_ARG;
+    if (lda < (a_order ? M : K) || ldb < (b_order ? N : K) || ldc < N) return MIPGEMM_ERR_INVALID_ARG;
+    const long long k_limit = (a_unsigned && b_unsigned) ? 33025 : ((a_unsigned || b_unsigned) ? 65793 : 131071);
+    if (K > k_limit) return MIPGEMM_ERR_K_TOO_LARGE;
+    if (!b_unsigned && !a_order && !b_order)
+        return gemm_impl(a_unsigned != 0, M, N, K, A, lda, static_cast<const int8_t*>(B), ldb, C, ldc, accumulate,
+                         stream_v, 0);
+    if (M == 0 || N == 0) {
+        tl_last_path = MIPGEMM_PATH_TRIVIAL;
+        return MIPGEMM_OK;
+    }
+    if (!C || reinterpret_cast<uintptr_t>(C) % 4 != 0 || (K > 0 && (!A || !B))) return MIPGEMM_ERR_INVALID_ARG;
+    DeviceState* dev = nullptr;
+    int st = get_device(&dev);
+    if (st != MIPGEMM_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    cudaError_t e;
+    if (K == 0) {
+        tl_last_path = MIPGEMM_PATH_TRIVIAL;
+        if (!accumulate) {
+            if ((e = launch_fill_zero(C, ldc, M, N, stream)) != cudaSuccess) return cuda_fail(e);
+            ++g_launches;
+        }
+        return MIPGEMM_OK;
+    }
+
+    // operands TMA cannot address go to K-contiguous scratch (plain or transposing re-pitch)
+    const long long pitch = round_up(K, 16);
+    const bool fix_a = !aligned16(A, lda), fix_b = !aligned16(B, ldb);
+    Scratch scratch(dev, stream);
+    size_t need = 0;
+    if (fix_a) need += align256(static_cast<size_t>(M) * pitch);
+    if (fix_b) need += align256(static_cast<size_t>(N) * pitch);
+    if ((st = scratch.reserve(need)) != MIPGEMM_OK) return st;
+    const void* a_use = A;
+    const void* b_use = B;
+    long long lda_use = lda, ldb_use = ldb;
+    int a_mn = a_order, b_mn = b_order, flags = 0;
+    if (fix_a) {
+        void* dst = scratch.take(static_cast<size_t>(M) * pitch);
+        e = a_order ? launch_transpose_repack(A, lda, dst, pitch, M, K, stream) : launch_repack(A, lda, dst, pitch, M, K, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+        ++g_launches;
+        a_use = dst; lda_use = pitch; a_mn = 0; flags |= MIPGEMM_PATH_REPACK;
+    }
+    if (fix_b) {
+        void* dst = scratch.take(static_cast<size_t>(N) * pitch);
+        e = b_order ? launch_transpose_repack(B, ldb, dst, pitch, N, K, stream) : launch_repack(B, ldb, dst, pitch, N, K, stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+        ++g_launches;
+        b_use = dst; ldb_use = pitch; b_mn = 0; flags |= MIPGEMM_PATH_REPACK;
+    }
+
+    const int block_k = 128;
+    const Plan pl = make_plan(M, N, K, block_k, dev, /*allow_pair=*/false, /*min_bn=*/b_mn ? 128 : 64);
+    DenseParams p;
+    std::memset(&p, 0, sizeof(p));
+    fill_common(p, pl, M, N, C, ldc, block_k, a_unsigned != 0, accumulate, dev);
+    p.a_mn = a_mn;
+    p.b_mn = b_mn;
+    p.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | ((b_unsigned ? 0u : 1u) << 10) |
+              (static_cast<uint32_t>(a_mn) << 15) | (static_cast<uint32_t>(b_mn) << 16) |
+              (static_cast<uint32_t>(pl.block_n >> 3) << 17) | (static_cast<uint32_t>(kBlockM >> 4) << 24);
+    // K-contiguous: tensor {K, rows}, box {128, tile rows}; M/N-contiguous: tensor {rows, K}, box {128, 128}
+    st = a_mn ? encode_tiled_2d(&p.tmap_a, a_use, M, K, lda_use, 128, block_k)
+              : encode_tiled_2d(&p.tmap_a, a_use, K, M, lda_use, block_k, kBlockM);
+    if (st != MIPGEMM_OK) return st;
+    st = b_mn ? encode_tiled_2d(&p.tmap_b, b_use, N, K, ldb_use, 128, block_k)
+              : encode_tiled_2d(&p.tmap_b, b_use, K, N, ldb_use, block_k, pl.block_n);
+    if (st != MIPGEMM_OK) return st;
+    if ((st = run_dense(p, pl, M, N, C, ldc, accumulate, dev, stream)) != MIPGEMM_OK) return st;
+    if (pl.split_k > 1) flags |= MIPGEMM_PATH_SPLITK;
+    tl_last_path = MIPGEMM_PATH_DENSE | flags;
+    return MIPGEMM_OK;
 }
 
 // Strided batch: C_b [+]= A_b * B_b for b < batch.  When every operand of every batch member is
@@ -878,6 +971,13 @@ int mipgemm_batched_u8s8s32(int64_t batch, int64_t M, int64_t N, int64_t K, cons
                             int64_t stride_a, const int8_t* B, int64_t ldb, int64_t stride_b, int32_t* C, int64_t ldc,
                             int64_t stride_c, int accumulate, void* stream) {
     return batched_impl(true, batch, M, N, K, A, lda, stride_a, B, ldb, stride_b, C, ldc, stride_c, accumulate, stream);
+}
+
+int mipgemm_gemm_ex(int a_unsigned, int b_unsigned, int a_order, int b_order, int c_col_major, int64_t M, int64_t N,
+                    int64_t K, const void* A, int64_t lda, const void* B, int64_t ldb, int32_t* C, int64_t ldc,
+                    int accumulate, void* stream) {
+    return gemm_ex_impl(a_unsigned, b_unsigned, a_order, b_order, c_col_major, M, N, K, A, lda, B, ldb, C, ldc,
+                        accumulate, stream);
 }
 
 uint64_t mipgemm_launch_count(void) { return g_launches.load(); }

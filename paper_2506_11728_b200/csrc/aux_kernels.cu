@@ -49,6 +49,35 @@ cudaError_t launch_repack(const void* src, long long src_pitch, void* dst, long 
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------- transposing repack
+// dst[i][k] = src[k*src_pitch + i] for i < rows_out, k < cols_out: turns an M- (or N-) contiguous
+// operand into the K-contiguous form the default path reads, through 32 x 32 byte tiles in shared
+// memory.  dst pitch is a multiple of 16; bytes beyond cols_out in a dst row are not written.
+__global__ void mip_transpose_repack_kernel(const uint8_t* __restrict__ src, long long src_pitch,
+                                            uint8_t* __restrict__ dst, long long dst_pitch,
+                                            long long rows_out, long long cols_out) {
+    __shared__ uint8_t tile[32][33];
+    const long long i0 = static_cast<long long>(blockIdx.x) * 32, k0 = static_cast<long long>(blockIdx.y) * 32;
+    for (int r = threadIdx.y; r < 32; r += blockDim.y) {          // r walks k, threadIdx.x walks i (contiguous)
+        const long long k = k0 + r, i = i0 + threadIdx.x;
+        tile[r][threadIdx.x] = (k < cols_out && i < rows_out) ? src[k * src_pitch + i] : 0;
+    }
+    __syncthreads();
+    for (int r = threadIdx.y; r < 32; r += blockDim.y) {          // r walks i, threadIdx.x walks k (contiguous)
+        const long long i = i0 + r, k = k0 + threadIdx.x;
+        if (i < rows_out && k < cols_out) dst[i * dst_pitch + k] = tile[threadIdx.x][r];
+    }
+}
+
+cudaError_t launch_transpose_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,
+                                    long long rows_out, long long cols_out, cudaStream_t stream) {
+    if (rows_out <= 0 || cols_out <= 0) return cudaSuccess;
+    const dim3 grid(static_cast<unsigned>((rows_out + 31) / 32), static_cast<unsigned>((cols_out + 31) / 32), 1);
+    mip_transpose_repack_kernel<<<grid, dim3(32, 8, 1), 0, stream>>>(
+        static_cast<const uint8_t*>(src), src_pitch, static_cast<uint8_t*>(dst), dst_pitch, rows_out, cols_out);
+    return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------- zero fill
 __global__ void mip_fill_zero_kernel(int32_t* C, long long ldc, long long M, long long N) {
     const long long total = M * N;

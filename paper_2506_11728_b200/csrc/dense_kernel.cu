@@ -335,6 +335,8 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                         tma_load_2d_pair(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta);
                     } else if (p.batch > 1) {
                         tma_load_3d(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta, tc.batch);
+                    } else if (p.a_mn) {      // tensor {M, K}: 128 bytes of M per k row
+                        tma_load_2d(a_dst, &p.tmap_a, full, m_cta, kb * p.block_k);
                     } else {
                         tma_load_2d(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta);
                     }
@@ -342,6 +344,10 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                         tma_load_2d_pair(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta);
                     else if (p.batch > 1)
                         tma_load_3d(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta, tc.batch);
+                    else if (p.b_mn)          // tensor {N, K}: one [k][128 B] block per 128 columns
+                        for (int blk = 0; blk * 128 < b_rows; ++blk)
+                            tma_load_2d(a_dst + a_bytes + blk * p.block_k * 128, &p.tmap_b, full, n_cta + blk * 128,
+                                        kb * p.block_k);
                     else
                         tma_load_2d(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta);
                 }
@@ -387,13 +393,17 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     if (t == 0 && kb == tc.kb_begin) MIP_STAMP(3);
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * stage_bytes;
-                    const uint64_t a_desc = make_kmajor_desc(a_addr, p.block_k);
-                    const uint64_t b_desc = make_kmajor_desc(a_addr + a_bytes, p.block_k);
+                    // K-major tiles advance 32 bytes per K = 32 step, MN-major tiles 32 rows of 128 bytes
+                    const uint64_t a_desc = p.a_mn ? make_mnmajor_desc(a_addr, p.block_k * 128)
+                                                   : make_kmajor_desc(a_addr, p.block_k);
+                    const uint64_t b_desc = p.b_mn ? make_mnmajor_desc(a_addr + a_bytes, p.block_k * 128)
+                                                   : make_kmajor_desc(a_addr + a_bytes, p.block_k);
+                    const uint64_t a_step = p.a_mn ? 256ull : 2ull, b_step = p.b_mn ? 256ull : 2ull;
                     const uint32_t empty_local = bar_empty + 8u * s;
                     const uint32_t empty_peer = kPair ? mapa_u32(empty_local, 1) : 0u;
                     if (elect_one()) {
                         for (uint32_t k = 0; k < k_steps; ++k) {
-                            mma_i8<kGroup>(d_tmem, a_desc + 2ull * k, b_desc + 2ull * k, p.idesc,
+                            mma_i8<kGroup>(d_tmem, a_desc + a_step * k, b_desc + b_step * k, p.idesc,
                                            (kb > tc.kb_begin || k > 0) ? 1u : 0u);
                         }
                         if (kPair) {

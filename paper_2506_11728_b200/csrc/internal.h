@@ -32,6 +32,7 @@ struct alignas(64) DenseParams {
     int stages;
     int tiles_m, tiles_n;
     int split_k, kb_per_split;
+    int a_mn, b_mn;          // 1: that operand is M- / N-contiguous in memory (k-block 128, one CTA per tile)
     int batch;               // > 1: strided batch; the tensor maps are rank 3 (z = batch index)
     long long stride_c;      // elements between consecutive C matrices of a batch
     int cluster_split;       // > 1: the split_k CTAs sharing a tile form a cluster and reduce through DSMEM
@@ -92,6 +93,8 @@ cudaError_t launch_skinny_ring(const SkinnyRingParams& p, int sm_count, cudaStre
 // Auxiliary kernels.
 cudaError_t launch_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,
                           long long rows, long long cols, cudaStream_t stream);
+cudaError_t launch_transpose_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,
+                                    long long rows_out, long long cols_out, cudaStream_t stream);
 cudaError_t launch_fill_zero(int32_t* C, long long ldc, long long M, long long N, cudaStream_t stream);
 struct Im2colParams {
     const uint8_t* X; uint8_t* out;

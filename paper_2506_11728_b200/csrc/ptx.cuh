@@ -298,6 +298,20 @@ __device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t smem_addr, uint32_
     return d;
 }
 
+// Same for an MN-major operand tile (the M or N index is the contiguous one): rows are k, each
+// row holds 128 bytes of M/N with the 128-byte TMA swizzle; 8-row groups are 1024 bytes apart
+// (stride byte offset), further 128-byte blocks of M/N are `block_bytes` apart (leading byte
+// offset).  One K = 32 step of the MMA spans four 8-row groups.
+__device__ __forceinline__ uint64_t make_mnmajor_desc(uint32_t smem_addr, uint32_t block_bytes) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);          // start address
+    d |= static_cast<uint64_t>((block_bytes >> 4) & 0x3FFFu) << 16;   // leading byte offset
+    d |= static_cast<uint64_t>(1024u >> 4) << 32;                     // stride byte offset
+    d |= static_cast<uint64_t>(1) << 46;                              // descriptor version (sm_100)
+    d |= 2ull << 61;                                                  // SWIZZLE_128B
+    return d;
+}
+
 // ---------------------------------------------------------------- global memory
 __device__ __forceinline__ void st_global_v8(int32_t* p, const uint32_t* v) {
     asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
