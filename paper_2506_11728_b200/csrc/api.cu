@@ -230,8 +230,8 @@ double plan_cost_us(int pair, int bn, int split, long long M, long long N, int k
     return 3.7 + (pair ? 1.0 : 0.0) + clk / 1900.0;   // pairs: cluster launch, two cluster barriers
 }
 
-Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceState* dev, bool allow_pair = true,
-               int min_bn = 64) {
+Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceState* dev, int min_bn = 64,
+               int min_bn_pair = 64) {
     const int sm_count = dev->sm_count;
     Plan pl{};
     pl.k_blocks = static_cast<int>((K + block_k - 1) / block_k);
@@ -243,15 +243,15 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
     double best = 1e30;
     // (an explicit split reduces int32 tiles in global memory, which a float output cannot share)
     const bool explicit_split = g_tuning.split_k != 0 && !tl_out_f32;
-    // (N-contiguous B tiles come in 128-column blocks: only 128 and 256 can be forced there)
-    const int forced_bn = (g_tuning.block_n && (min_bn <= 64 || g_tuning.block_n % 128 == 0)) ? g_tuning.block_n : 0;
+    // (N-contiguous B tiles come in 128-column blocks per CTA: a forced width must respect that)
+    const int forced_bn = (g_tuning.block_n && (min_bn <= 64 || g_tuning.block_n == 256)) ? g_tuning.block_n : 0;
     for (int pair = 0; pair <= 1; ++pair) {
-        if (pair && (dev->pair_clusters <= 0 || !allow_pair)) continue;
+        if (pair && dev->pair_clusters <= 0) continue;
         if (g_tuning.force_path == MIPGEMM_PATH_DENSE_PAIR && !pair && dev->pair_clusters > 0) continue;
         if (g_tuning.force_path == MIPGEMM_PATH_DENSE && pair) continue;
         for (int bn = 64; bn <= 256; bn *= 2) {
             int bn_use = bn;
-            if (bn < min_bn) continue;
+            if (bn < (pair ? min_bn_pair : min_bn)) continue;
             if (forced_bn) {
                 if (bn != 256) continue;                      // a single candidate: the forced width
                 bn_use = forced_bn;
@@ -623,7 +623,9 @@ int gemm_ex_impl(int a_unsigned, int b_unsigned, int a_order, int b_order, int c
     }
 
     const int block_k = 128;
-    const Plan pl = make_plan(M, N, K, block_k, dev, /*allow_pair=*/false, /*min_bn=*/b_mn ? 128 : 64);
+    // N-contiguous B is staged in blocks of 128 columns per CTA: 128 or 256 wide tiles for one
+    // CTA, 256 wide for a pair (each CTA stages half)
+    const Plan pl = make_plan(M, N, K, block_k, dev, b_mn ? 128 : 64, b_mn ? 256 : 64);
     DenseParams p;
     std::memset(&p, 0, sizeof(p));
     fill_common(p, pl, M, N, C, ldc, block_k, a_unsigned != 0, accumulate, dev);
@@ -631,17 +633,18 @@ int gemm_ex_impl(int a_unsigned, int b_unsigned, int a_order, int b_order, int c
     p.b_mn = b_mn;
     p.idesc = (2u << 4) | ((a_unsigned ? 0u : 1u) << 7) | ((b_unsigned ? 0u : 1u) << 10) |
               (static_cast<uint32_t>(a_mn) << 15) | (static_cast<uint32_t>(b_mn) << 16) |
-              (static_cast<uint32_t>(pl.block_n >> 3) << 17) | (static_cast<uint32_t>(kBlockM >> 4) << 24);
+              (static_cast<uint32_t>(pl.block_n >> 3) << 17) |
+              (static_cast<uint32_t>((pl.pair ? 2 * kBlockM : kBlockM) >> 4) << 24);
     // K-contiguous: tensor {K, rows}, box {128, tile rows}; M/N-contiguous: tensor {rows, K}, box {128, 128}
     st = a_mn ? encode_tiled_2d(&p.tmap_a, a_use, M, K, lda_use, 128, block_k)
               : encode_tiled_2d(&p.tmap_a, a_use, K, M, lda_use, block_k, kBlockM);
     if (st != MIPGEMM_OK) return st;
     st = b_mn ? encode_tiled_2d(&p.tmap_b, b_use, N, K, ldb_use, 128, block_k)
-              : encode_tiled_2d(&p.tmap_b, b_use, K, N, ldb_use, block_k, pl.block_n);
+              : encode_tiled_2d(&p.tmap_b, b_use, K, N, ldb_use, block_k, pl.pair ? pl.block_n / 2 : pl.block_n);
     if (st != MIPGEMM_OK) return st;
     if ((st = run_dense(p, pl, M, N, C, ldc, accumulate, dev, stream)) != MIPGEMM_OK) return st;
     if (pl.split_k > 1) flags |= MIPGEMM_PATH_SPLITK;
-    tl_last_path = MIPGEMM_PATH_DENSE | flags;
+    tl_last_path = (pl.pair ? MIPGEMM_PATH_DENSE_PAIR : MIPGEMM_PATH_DENSE) | flags;
     return MIPGEMM_OK;
 }
 

@@ -209,7 +209,7 @@ __device__ __forceinline__ void coalesced_chunk(const DenseParams& p, uint32_t b
     }
 }
 
-template <bool kPair>
+template <bool kPair, bool kMN>
 __global__ void __launch_bounds__(kDenseThreads, 1)
 mip_dense_kernel(const __grid_constant__ DenseParams p) {
     constexpr int kGroup = kPair ? 2 : 1;
@@ -331,25 +331,29 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                             tma_load_im2col_4d(a_dst, &p.tmap_a, full, cc * p.block_k, cw, chh, cn,
                                                static_cast<uint16_t>(fs * p.dil_w),
                                                static_cast<uint16_t>(fr * p.dil_h));
+                    } else if (kMN && p.a_mn) {   // tensor {M, K}: 128 bytes of M per k row
+                        if (kPair) tma_load_2d_pair(a_dst, &p.tmap_a, full, m_cta, kb * p.block_k);
+                        else tma_load_2d(a_dst, &p.tmap_a, full, m_cta, kb * p.block_k);
                     } else if (kPair) {
                         tma_load_2d_pair(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta);
                     } else if (p.batch > 1) {
                         tma_load_3d(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta, tc.batch);
-                    } else if (p.a_mn) {      // tensor {M, K}: 128 bytes of M per k row
-                        tma_load_2d(a_dst, &p.tmap_a, full, m_cta, kb * p.block_k);
                     } else {
                         tma_load_2d(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta);
                     }
-                    if (kPair)
+                    if (kMN && p.b_mn) {          // tensor {N, K}: one [k][128 B] block per 128 columns
+                        for (int blk = 0; blk * 128 < b_rows; ++blk) {
+                            const uint32_t dst = a_dst + a_bytes + blk * p.block_k * 128;
+                            if (kPair) tma_load_2d_pair(dst, &p.tmap_b, full, n_cta + blk * 128, kb * p.block_k);
+                            else tma_load_2d(dst, &p.tmap_b, full, n_cta + blk * 128, kb * p.block_k);
+                        }
+                    } else if (kPair) {
                         tma_load_2d_pair(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta);
-                    else if (p.batch > 1)
+                    } else if (p.batch > 1) {
                         tma_load_3d(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta, tc.batch);
-                    else if (p.b_mn)          // tensor {N, K}: one [k][128 B] block per 128 columns
-                        for (int blk = 0; blk * 128 < b_rows; ++blk)
-                            tma_load_2d(a_dst + a_bytes + blk * p.block_k * 128, &p.tmap_b, full, n_cta + blk * 128,
-                                        kb * p.block_k);
-                    else
+                    } else {
                         tma_load_2d(a_dst + a_bytes, &p.tmap_b, full, kb * p.block_k, n_cta);
+                    }
                 }
                 if (issued == 0) MIP_STAMP(2);
                 if (p.a_im2col && ++cc == p.c_chunks) {   // next filter tap (r, s)
@@ -394,11 +398,12 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * stage_bytes;
                     // K-major tiles advance 32 bytes per K = 32 step, MN-major tiles 32 rows of 128 bytes
-                    const uint64_t a_desc = p.a_mn ? make_mnmajor_desc(a_addr, p.block_k * 128)
-                                                   : make_kmajor_desc(a_addr, p.block_k);
-                    const uint64_t b_desc = p.b_mn ? make_mnmajor_desc(a_addr + a_bytes, p.block_k * 128)
-                                                   : make_kmajor_desc(a_addr + a_bytes, p.block_k);
-                    const uint64_t a_step = p.a_mn ? 256ull : 2ull, b_step = p.b_mn ? 256ull : 2ull;
+                    const bool a_mn = kMN && p.a_mn, b_mn = kMN && p.b_mn;
+                    const uint64_t a_desc = a_mn ? make_mnmajor_desc(a_addr, p.block_k * 128)
+                                                 : make_kmajor_desc(a_addr, p.block_k);
+                    const uint64_t b_desc = b_mn ? make_mnmajor_desc(a_addr + a_bytes, p.block_k * 128)
+                                                 : make_kmajor_desc(a_addr + a_bytes, p.block_k);
+                    const uint64_t a_step = a_mn ? 256ull : 2ull, b_step = b_mn ? 256ull : 2ull;
                     const uint32_t empty_local = bar_empty + 8u * s;
                     const uint32_t empty_peer = kPair ? mapa_u32(empty_local, 1) : 0u;
                     if (elect_one()) {
@@ -585,11 +590,18 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 }
 
 cudaError_t dense_init() {
-    cudaError_t e = cudaFuncSetAttribute(mip_dense_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kSmemBudget);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(mip_dense_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                kSmemBudget);
+    cudaError_t e = cudaFuncSetAttribute(mip_dense_kernel<false, false>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(mip_dense_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(mip_dense_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(mip_dense_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget);
+    return e;
 }
 
 // All launches allow programmatic stream serialisation (see pdl_wait() in the kernel).
@@ -608,7 +620,10 @@ cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cuda
     pdl_attribute(attr[0]);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false>, p);
+    // (the M-/N-contiguous operand forms live in an instantiation of their own, so the common
+    // kernel's issue loops carry none of their address arithmetic)
+    if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, true>, p);
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false>, p);
 }
 
 // One-CTA-per-tile kernel launched in clusters of `cluster` CTAs (cluster split-K); `grid` is a
@@ -628,7 +643,7 @@ cudaError_t launch_dense_cluster(const DenseParams& p, int grid, int cluster, si
     pdl_attribute(attr[1]);
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false>, p);
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false>, p);
 }
 
 // `grid` counts CTAs and must be even: consecutive CTAs form a cluster of two.
@@ -646,7 +661,8 @@ cudaError_t launch_dense_pair(const DenseParams& p, int grid, size_t smem_bytes,
     pdl_attribute(attr[1]);
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true>, p);
+    if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, true>, p);
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, false>, p);
 }
 
 // Largest number of co-resident 2-CTA clusters for the pair kernel (0 on failure).
@@ -663,7 +679,7 @@ int dense_pair_max_clusters(size_t smem_bytes) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, mip_dense_kernel<true>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, mip_dense_kernel<true, false>, &cfg) != cudaSuccess) {
         (void)cudaGetLastError();
         return 0;
     }

@@ -60,6 +60,22 @@ def test_storage_orders_aligned(mg, ao, bo):
     run_ex(mg, 1, 0, ao, bo, 0, 640, 384, 272, accumulate=True, seed=33)
 
 
+@pytest.mark.parametrize("ao,bo", [(0, 1), (1, 0), (1, 1)])
+def test_storage_orders_on_both_kernel_forms(mg, ao, bo):
+    """One CTA per tile and CTA pairs, tile widths 128 and 256, split K."""
+    try:
+        for force, bn in [(mg.PATH_DENSE, 128), (mg.PATH_DENSE, 256), (mg.PATH_DENSE_PAIR, 256), (mg.PATH_DENSE, 0)]:
+            mg.mipgemm_set_tuning(block_n=bn, force_path=force)
+            p = run_ex(mg, 1, 1, ao, bo, 0, 528, 784, 400, seed=90 + 2 * ao + bo)
+            assert p & force and not p & mg.PATH_REPACK
+            run_ex(mg, 0, 0, ao, bo, 0, 272, 144, 1024, accumulate=True, pad=(16, 32, 0), seed=95 + 2 * ao + bo)
+        mg.mipgemm_set_tuning(split_k=3, force_path=mg.PATH_DENSE)
+        p = run_ex(mg, 0, 1, ao, bo, 0, 208, 304, 2048, seed=99)
+        assert p & mg.PATH_SPLITK
+    finally:
+        mg.mipgemm_set_tuning()
+
+
 @pytest.mark.parametrize("au,bu", list(itertools.product([0, 1], [0, 1])))
 def test_signedness_pairs(mg, au, bu):
     run_ex(mg, au, bu, 0, 0, 0, 300, 260, 400, seed=40 + 2 * au + bu)
