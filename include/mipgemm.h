@@ -38,9 +38,9 @@
  *
  * Scratch memory
  * --------------
- * Some calls need global scratch memory (operand re-pitching, the explicit
- * im2col matrix for convolutions the tensor-memory-accelerator cannot gather,
- * split-K partial sums).  By default it is taken with cudaMallocAsync on the
+ * Some calls need global scratch memory (operand re-pitching, slot-padded
+ * filters for convolutions gathered in software, the explicit im2col matrix
+ * for the few convolutions neither the TMA nor the gather warps can handle).  By default it is taken with cudaMallocAsync on the
  * call's stream and released with cudaFreeAsync after the last kernel of the
  * call.  A caller may instead lend a buffer with mipgemm_set_workspace(); calls
  * that need more than was lent fail with MIPGEMM_ERR_WORKSPACE.  A lent buffer
@@ -79,7 +79,8 @@ typedef enum {
     MIPGEMM_PATH_SPLITK = 0x200,  /* flag: K was split and reduced with integer atomics      */
     MIPGEMM_PATH_IM2COL_TMA = 0x400,   /* flag: conv gathered by TMA im2col loads            */
     MIPGEMM_PATH_IM2COL_EXPLICIT = 0x800, /* flag: conv materialised the augmented matrix    */
-    MIPGEMM_PATH_BATCHED = 0x1000      /* flag: a whole strided batch ran as one launch       */
+    MIPGEMM_PATH_BATCHED = 0x1000,     /* flag: a whole strided batch ran as one launch       */
+    MIPGEMM_PATH_IM2COL_GATHER = 0x2000 /* flag: conv gathered into shared memory by extra warps */
 } mipgemm_path_t;
 
 /*

@@ -30,6 +30,7 @@ PATH_NONE, PATH_DENSE, PATH_DENSE_PAIR, PATH_SKINNY, PATH_TRIVIAL = range(5)
 PATH_MASK = 0xFF
 PATH_REPACK, PATH_SPLITK, PATH_IM2COL_TMA, PATH_IM2COL_EXPLICIT = 0x100, 0x200, 0x400, 0x800
 PATH_BATCHED = 0x1000
+PATH_IM2COL_GATHER = 0x2000
 
 #: every symbol include/mipgemm.h declares, with (restype, argtypes)
 SIGNATURES = {

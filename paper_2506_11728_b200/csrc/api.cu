@@ -231,7 +231,7 @@ double plan_cost_us(int pair, int bn, int split, long long M, long long N, int k
 }
 
 Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceState* dev, int min_bn = 64,
-               int min_bn_pair = 64) {
+               int min_bn_pair = 64, bool one_cta_no_split = false) {
     const int sm_count = dev->sm_count;
     Plan pl{};
     pl.k_blocks = static_cast<int>((K + block_k - 1) / block_k);
@@ -246,7 +246,7 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
     // (N-contiguous B tiles come in 128-column blocks per CTA: a forced width must respect that)
     const int forced_bn = (g_tuning.block_n && (min_bn <= 64 || g_tuning.block_n == 256)) ? g_tuning.block_n : 0;
     for (int pair = 0; pair <= 1; ++pair) {
-        if (pair && dev->pair_clusters <= 0) continue;
+        if (pair && (dev->pair_clusters <= 0 || one_cta_no_split)) continue;
         if (g_tuning.force_path == MIPGEMM_PATH_DENSE_PAIR && !pair && dev->pair_clusters > 0) continue;
         if (g_tuning.force_path == MIPGEMM_PATH_DENSE && pair) continue;
         for (int bn = 64; bn <= 256; bn *= 2) {
@@ -261,7 +261,7 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
             const long long tiles = ((M + rows - 1) / rows) * ((N + bn_use - 1) / bn_use);
             for (int split = 1; split <= 8; split *= 2) {
                 if (split > 1) {
-                    if (pair || explicit_split || g_tuning_no_cluster_split) break;
+                    if (pair || explicit_split || g_tuning_no_cluster_split || one_cta_no_split) break;
                     if (tiles * split > sm_count || bn_use / split < 32 || (bn_use / split) % 32 != 0) break;
                     if (pl.k_blocks / split < 2) break;
                 }
@@ -288,14 +288,14 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
     if (stages < 2) stages = 2;
     pl.stages = stages;
 
-    int split = explicit_split ? g_tuning.split_k : best_split;
+    int split = (explicit_split && !one_cta_no_split) ? g_tuning.split_k : best_split;
     if (pl.pair) split = 1;
     if (split > pl.k_blocks) split = pl.k_blocks;
     if (split < 1) split = 1;
     // the automatic split is a cluster split (DSMEM reduce-scatter: the receive buffers must fit
     // the idle pipeline stages); an explicit factor uses zero fill + TMA tile reduce-add
     pl.cluster_split = 0;
-    if (!explicit_split && split > 1) {
+    if (!(explicit_split && !one_cta_no_split) && split > 1) {
         if (512LL * bn * (split - 1) / split <= static_cast<long long>(stages) * stage_bytes) pl.cluster_split = split;
         else split = 1;
     }
@@ -394,7 +394,7 @@ int run_dense(DenseParams& p, const Plan& pl, long long M, long long N, int32_t*
         e = launch_dense_cluster(p, static_cast<int>(units), pl.cluster_split, smem, stream);
     } else {
         const int grid = static_cast<int>(units < dev->sm_count ? units : dev->sm_count);
-        e = launch_dense(p, grid, smem, stream);
+        e = p.a_gather ? launch_dense_gather(p, grid, smem, stream) : launch_dense(p, grid, smem, stream);
     }
     ++g_launches;
     if (e != cudaSuccess) return cuda_fail(e);
@@ -553,6 +553,20 @@ bool conv_tma_eligible(const ConvGeom& g, const void* X, const void* Wt) {
     if ((g.S - 1) * g.dil_w > 65535 || (g.R - 1) * g.dil_h > 65535) return false;
     if (g.W >= (1LL << 31) || g.H >= (1LL << 31) || g.Nb >= (1LL << 31)) return false;
     if (g.H * g.W * g.Cin >= (1LL << 40)) return false;
+    return true;
+}
+
+// Convolutions TMA cannot gather (channel count not a multiple of 64, e.g. an RGB stem) whose
+// filter rows are contiguous in the image (dil_w == 1): operand A is built in shared memory
+// by eight extra warps of the dense kernel, so the augmented matrix never exists in memory.
+bool conv_gather_eligible(const ConvGeom& g) {
+    if (g.dil_w != 1) return false;
+    const long long seg = static_cast<long long>(g.S) * g.Cin;
+    const long long slot = round_up(seg, 16);
+    if (slot * g.R > 8192) return false;                       // whole rows of A stay short
+    if (g.W * g.Cin >= (1LL << 30) || g.H >= (1LL << 30)) return false;
+    const long long xbytes = g.Nb * g.H * g.W * g.Cin;
+    if (xbytes < 64 || xbytes >= (1LL << 30)) return false;    // (32-bit byte offsets; loads assume some size)
     return true;
 }
 
@@ -861,6 +875,41 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
         return MIPGEMM_OK;
     }
 
+    if (conv_gather_eligible(g) && g_tuning.force_path != MIPGEMM_PATH_IM2COL_EXPLICIT) {
+        const int seg = S * static_cast<int>(Cin);
+        const int slot = static_cast<int>(round_up(seg, 16));
+        const long long Kp = static_cast<long long>(R) * slot;      // K with every filter row padded to its slot
+        const int block_k = 128;
+        Scratch scratch(dev, stream);
+        if ((st = scratch.reserve(align256(static_cast<size_t>(Cout) * Kp))) != MIPGEMM_OK) return st;
+        int8_t* wp = static_cast<int8_t*>(scratch.take(static_cast<size_t>(Cout) * Kp));
+        cudaError_t e = launch_weight_slots(Wt, wp, Cout, R, seg, slot, stream);
+        ++g_launches;
+        if (e != cudaSuccess) return cuda_fail(e);
+        const Plan pl = make_plan(M, Cout, Kp, block_k, dev, 64, 64, /*one_cta_no_split=*/true);
+        DenseParams p;
+        std::memset(&p, 0, sizeof(p));
+        fill_common(p, pl, M, Cout, Y, Cout, block_k, true, accumulate, dev);
+        p.a_gather = 1;
+        p.gx = X;
+        p.g_xbytes = g.Nb * g.H * g.W * g.Cin;
+        p.g_h = static_cast<int>(g.H);
+        p.g_row_bytes = static_cast<int>(g.W * g.Cin);
+        p.g_cin = static_cast<int>(g.Cin);
+        p.g_seg = seg;
+        p.g_slot = slot;
+        p.g_chunks = static_cast<int>(Kp / 16);
+        p.conv_wo = static_cast<int>(g.Wo);
+        p.conv_howo = static_cast<int>(g.Ho * g.Wo);
+        p.stride_w = stride_w; p.stride_h = stride_h;
+        p.pad_w = pad_w; p.pad_h = pad_h;
+        p.dil_w = dil_w; p.dil_h = dil_h;
+        if ((st = encode_tiled_2d(&p.tmap_b, wp, Kp, Cout, Kp, block_k, pl.block_n)) != MIPGEMM_OK) return st;
+        if ((st = run_dense(p, pl, M, Cout, Y, Cout, accumulate, dev, stream)) != MIPGEMM_OK) return st;
+        tl_last_path = MIPGEMM_PATH_DENSE | MIPGEMM_PATH_IM2COL_GATHER;
+        return MIPGEMM_OK;
+    }
+
     // Explicit lowering: materialise the augmented matrix (zero-padded to a 16-byte pitch),
     // then run the GEMM on it.  The weight matrix is re-pitched by the GEMM if K % 16 != 0.
     const long long k_pitch = round_up(K, 16);
@@ -922,6 +971,7 @@ size_t mipgemm_workspace_query_conv(int64_t Nb, int64_t H, int64_t W, int64_t Ci
     const long long M = g.Nb * g.Ho * g.Wo;
     if (conv_is_pointwise(g)) return gemm_scratch_bytes(M, Cout, Cin, nullptr, Cin, nullptr, Cin);
     if (conv_tma_eligible(g, nullptr, nullptr)) return 0;
+    if (conv_gather_eligible(g)) return align256(static_cast<size_t>(Cout) * R * round_up(static_cast<long long>(S) * Cin, 16));
     const long long K = static_cast<long long>(R) * S * Cin;
     const long long k_pitch = round_up(K, 16);
     return align256(static_cast<size_t>(M) * k_pitch) + gemm_scratch_bytes(M, Cout, K, nullptr, k_pitch, nullptr, K);

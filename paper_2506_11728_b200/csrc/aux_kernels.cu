@@ -88,6 +88,35 @@ __global__ void mip_fill_zero_kernel(int32_t* C, long long ldc, long long M, lon
     }
 }
 
+__global__ void mip_weight_slots_kernel(const int8_t* __restrict__ src, int8_t* __restrict__ dst, long long total,
+                                        int R, int seg, int slot) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= total) return;
+    const int b = static_cast<int>(i % slot);
+    const long long rr = i / slot;               // row * R + r
+    dst[i] = b < seg ? src[rr * seg + b] : static_cast<int8_t>(0);
+}
+
+cudaError_t launch_weight_slots(const int8_t* src, int8_t* dst, long long rows, int R, int seg, int slot,
+                                cudaStream_t stream) {
+    const long long total = rows * R * slot;
+    if (total == 0) return cudaSuccess;
+    const int threads = 256;
+    const long long blocks = (total + threads - 1) / threads;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+    cfg.blockDim = dim3(threads, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, mip_weight_slots_kernel, src, dst, total, R, seg, slot);
+}
+
 cudaError_t launch_fill_zero(int32_t* C, long long ldc, long long M, long long N, cudaStream_t stream) {
     if (M <= 0 || N <= 0) return cudaSuccess;
     const int threads = 256;

@@ -209,8 +209,51 @@ __device__ __forceinline__ void coalesced_chunk(const DenseParams& p, uint32_t b
     }
 }
 
-template <bool kPair, bool kMN>
-__global__ void __launch_bounds__(kDenseThreads, 1)
+// Gather form: one 16-byte chunk of a row of A is copied from the image with five 4-byte loads
+// at the source address rounded down; funnel shifts then bring the sixteen bytes into place.
+// The two rare cases are kept off the common path, which stays
+// a handful of instructions per chunk -- the gather warps are bound by their instruction latency:
+//   * the pixel's window hangs over the left or right edge of the image: the bytes outside
+//     [keep_lo, keep_hi) of the chunk (taps outside the image) are cleared with gather_mask;
+//   * gather_border_chunk: the chunk begins before the batch or reaches past its end (first and
+//     last pixels of the whole batch only).  It is assembled byte by byte from the bytes that
+//     exist; all others are either taps outside the image (zero) or meet a zero weight.
+// (volatile loads: the loads of a k-block stay ahead of the first shared-memory store, i.e. all
+// in flight together, instead of each being sunk to its use)
+__device__ __forceinline__ uint32_t ldg_nc_u32(const uint32_t* ptr) {
+    uint32_t v;
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(ptr));
+    return v;
+}
+
+// Byte mask of a 16-byte chunk that keeps bytes [keep_lo, keep_hi) (any integers; clamped here).
+__device__ __forceinline__ uint4 gather_mask(int keep_lo, int keep_hi) {
+    uint32_t w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t a = static_cast<uint32_t>(min(max(keep_lo - 4 * j, 0), 4)) * 8u;   // bits to clear from below
+        const uint32_t b = static_cast<uint32_t>(min(max(keep_hi - 4 * j, 0), 4)) * 8u;   // bits to keep from below
+        // (clamped funnel shift: 0xFFFFFFFF << n, and 0 for n = 32)
+        w[j] = __funnelshift_lc(0u, 0xFFFFFFFFu, a) & ~__funnelshift_lc(0u, 0xFFFFFFFFu, b);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__device__ __noinline__ void gather_border_chunk(const uint8_t* gx, int xbytes, int src, int keep_lo, int keep_hi,
+                                                 uint32_t smem_dst) {
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+    for (int t = 0; t < 16; ++t) {
+        const int i = src + t;
+        if (t >= keep_lo && t < keep_hi && i >= 0 && i < xbytes) {
+            const uint32_t byte = static_cast<uint32_t>(gx[i]) << (8 * (t & 3));
+            if (t < 4) w[0] |= byte; else if (t < 8) w[1] |= byte; else if (t < 12) w[2] |= byte; else w[3] |= byte;
+        }
+    }
+    st_shared_v4(smem_dst, w);
+}
+
+template <bool kPair, bool kMN, bool kGather>
+__global__ void __launch_bounds__(kGather ? kGatherThreads : kDenseThreads, 1)
 mip_dense_kernel(const __grid_constant__ DenseParams p) {
     constexpr int kGroup = kPair ? 2 : 1;
     constexpr int kRowsPerTile = kPair ? 2 * kBlockM : kBlockM;
@@ -250,7 +293,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(bar_full + 8u * s, 1);
+            mbar_init(bar_full + 8u * s, kGather ? 9 : 1);   // + one arrival per gather warp
             mbar_init(bar_empty + 8u * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -260,7 +303,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         mbar_init(bar_drain, 1);
         *abort_flag = 0;
         fence_mbar_init();
-        tma_prefetch_desc(&p.tmap_a);
+        if (!kGather) tma_prefetch_desc(&p.tmap_a);
         tma_prefetch_desc(&p.tmap_b);
         if (p.c_mode == 1 || p.c_mode == 2) tma_prefetch_desc(&p.tmap_c);
     }
@@ -290,7 +333,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         // ------------------------------------------------------------ TMA producer (whole warp loops)
         uint32_t s = 0, phase = 0, issued = 0;
         bool ok = true;
-        const uint32_t tx_bytes = kPair ? 2u * stage_bytes : stage_bytes;
+        const uint32_t tx_bytes = kGather ? b_bytes : (kPair ? 2u * stage_bytes : stage_bytes);
         for (int unit = first_unit; unit < total_units && ok; unit += unit_stride) {
             const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
             const int m_cta = tc.m0 + static_cast<int>(cta_rank) * kBlockM;
@@ -322,7 +365,9 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 const uint32_t a_dst = smem_base + s * stage_bytes;
                 if (elect_one()) {
                     if (leader) mbar_arrive_expect_tx(full_local, tx_bytes);
-                    if (p.a_im2col) {
+                    if (kGather) {
+                        // operand A is written by the gather warps
+                    } else if (p.a_im2col) {
                         if (kPair)
                             tma_load_im2col_4d_pair(a_dst, &p.tmap_a, full, cc * p.block_k, cw, chh, cn,
                                                     static_cast<uint16_t>(fs * p.dil_w),
@@ -445,7 +490,123 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 }
             }
         }
-    } else {
+    } else if (kGather && warp >= 8) {
+        // ------------------------------------------------------------ software im2col (8 warps)
+        // Thread = every second 16-byte chunk of one row of the tile (one output pixel): warps
+        // 8-11 take the even chunks of rows 0-127, warps 12-15 the odd ones.  For every k-block a
+        // thread writes its (up to) four chunks into the stage in the 128-byte-swizzled K-major
+        // layout the TMA would have produced, makes them visible to the tensor core's proxy and
+        // arrives.  The loads of the next k-block (of this or the next tile) are issued before the
+        // current one is shifted and stored, so their latency is hidden.  Byte offsets into the
+        // batch fit 31 bits (checked by the host).
+        const int row = ((warp - 8) & 3) * 32 + lane;
+        const int parity = (warp - 8) >> 2;
+        const int xbytes = static_cast<int>(p.g_xbytes);
+        const uint32_t align = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(p.gx)) & 3u;
+        constexpr int kNone = -0x40000000;
+        struct Item {                 // one k-block of one tile, as seen by this thread
+            int src[4], offs[4];      // source byte offset of each chunk (kNone: all zero), offset in its slot
+            int lo, hi, q0;
+            bool edge;
+            uint4 mask;               // slots of 16 or 32 bytes: every chunk of this thread has the same offset
+            uint32_t x[4][5];
+        };
+        const bool fixed_off = p.g_slot <= 32;
+        // per-tile state of the tile that `prepare` is walking through
+        int unit = first_unit, kb = 0, kb_end = 0;
+        int h0 = 0, lo = 0, hi = 0, src0 = 0;
+        bool edge = false;
+        auto next_item = [&](Item& it) -> bool {     // false: no more work
+            while (kb >= kb_end) {
+                if (unit >= total_units) return false;
+                const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
+                unit += unit_stride;
+                kb = tc.kb_begin;
+                kb_end = tc.kb_end;
+                const int m = tc.m0 + row;
+                const int mm = m < p.M ? m : 0;
+                const int n_img = mm / p.conv_howo;
+                const int rem = mm - n_img * p.conv_howo;
+                const int ho = rem / p.conv_wo;
+                const int wo = rem - ho * p.conv_wo;
+                // rows beyond M: every filter row falls outside the image, the row of A is zero
+                h0 = m < p.M ? ho * p.stride_h - p.pad_h : kNone;
+                const int wb = (wo * p.stride_w - p.pad_w) * p.g_cin;   // window start, bytes into the image row
+                // taps inside the image row: bytes [lo, hi) of every slot.  When nothing is cut off on
+                // the right, the slot's padding bytes are copied as they come (they meet zero weights).
+                lo = max(0, -wb);
+                hi = (p.g_row_bytes - wb >= p.g_seg) ? p.g_slot : p.g_row_bytes - wb;
+                edge = lo > 0 || hi < p.g_slot;
+                src0 = n_img * p.g_h * p.g_row_bytes + wb;
+            }
+            it.lo = lo; it.hi = hi; it.edge = edge;
+            it.q0 = kb * 8 + parity;
+            int r = (it.q0 * 16) / p.g_slot;
+            int off = it.q0 * 16 - r * p.g_slot;
+            it.mask = gather_mask(lo - off, hi - off);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int h = h0 + r * p.dil_h;
+                const bool use = it.q0 + 2 * c < p.g_chunks && off < p.g_seg &&
+                                 static_cast<unsigned>(h) < static_cast<unsigned>(p.g_h) && off < hi && off + 16 > lo;
+                it.src[c] = use ? src0 + h * p.g_row_bytes + off : kNone;
+                it.offs[c] = off;
+                off += 32;
+                while (off >= p.g_slot) { off -= p.g_slot; ++r; }
+            }
+            // all loads back to back and unconditional (chunks that are all zero, and the few at the
+            // very ends of the batch, load the batch's first words instead)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const bool plain = it.src[c] >= 4 && it.src[c] <= xbytes - 24;
+                const uint32_t* w = reinterpret_cast<const uint32_t*>(
+                    (reinterpret_cast<uintptr_t>(p.gx) + static_cast<uintptr_t>(plain ? it.src[c] : 4)) &
+                    ~static_cast<uintptr_t>(3));
+#pragma unroll
+                for (int j = 0; j < 5; ++j) it.x[c][j] = ldg_nc_u32(w + j);
+            }
+            ++kb;
+            return true;
+        };
+        uint32_t s = 0, phase = 0;
+        Item cur, nxt;
+        bool have = next_item(cur);
+        while (have) {
+            const bool have_next = next_item(nxt);
+            if (!mbar_wait(bar_empty + 8u * s, phase ^ 1u, abort_flag, budget)) break;
+            const uint32_t dst = smem_base + s * stage_bytes + static_cast<uint32_t>(row) * 128u;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if (cur.q0 + 2 * c < p.g_chunks) {
+                    const uint32_t at = dst + (static_cast<uint32_t>((parity + 2 * c) ^ (row & 7)) << 4);
+                    const int sc = cur.src[c];
+                    if (sc != kNone && !(sc >= 4 && sc <= xbytes - 24)) {   // at the very ends of the batch
+                        gather_border_chunk(p.gx, xbytes, sc, cur.lo - cur.offs[c], cur.hi - cur.offs[c], at);
+                    } else {
+                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                        if (sc != kNone) {
+                            const uint32_t sh = ((static_cast<uint32_t>(sc) + align) & 3u) * 8u;
+                            v.x = __funnelshift_r(cur.x[c][0], cur.x[c][1], sh);
+                            v.y = __funnelshift_r(cur.x[c][1], cur.x[c][2], sh);
+                            v.z = __funnelshift_r(cur.x[c][2], cur.x[c][3], sh);
+                            v.w = __funnelshift_r(cur.x[c][3], cur.x[c][4], sh);
+                            uint4 mk = cur.mask;
+                            if (!fixed_off && cur.edge) mk = gather_mask(cur.lo - cur.offs[c], cur.hi - cur.offs[c]);
+                            v.x &= mk.x; v.y &= mk.y; v.z &= mk.z; v.w &= mk.w;
+                        }
+                        uint32_t vv[4] = {v.x, v.y, v.z, v.w};
+                        st_shared_v4(at, vv);
+                    }
+                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_full + 8u * s);
+            if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
+            cur = nxt;
+            have = have_next;
+        }
+    } else if (warp < 6) {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;
         int t = 0;
@@ -590,16 +751,19 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 }
 
 cudaError_t dense_init() {
-    cudaError_t e = cudaFuncSetAttribute(mip_dense_kernel<false, false>,
+    cudaError_t e = cudaFuncSetAttribute(mip_dense_kernel<false, false, false>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(mip_dense_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(mip_dense_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(mip_dense_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(mip_dense_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(mip_dense_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(mip_dense_kernel<true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(mip_dense_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget);
     return e;
 }
@@ -622,8 +786,22 @@ cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cuda
     cfg.numAttrs = 1;
     // (the M-/N-contiguous operand forms live in an instantiation of their own, so the common
     // kernel's issue loops carry none of their address arithmetic)
-    if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, true>, p);
-    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false>, p);
+    if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, true, false>, p);
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, false>, p);
+}
+
+// One CTA per tile with eight additional warps that gather operand A from an image batch.
+cudaError_t launch_dense_gather(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+    cfg.blockDim = dim3(kGatherThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    pdl_attribute(attr[0]);
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, true>, p);
 }
 
 // One-CTA-per-tile kernel launched in clusters of `cluster` CTAs (cluster split-K); `grid` is a
@@ -643,7 +821,7 @@ cudaError_t launch_dense_cluster(const DenseParams& p, int grid, int cluster, si
     pdl_attribute(attr[1]);
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false>, p);
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, false>, p);
 }
 
 // `grid` counts CTAs and must be even: consecutive CTAs form a cluster of two.
@@ -661,8 +839,8 @@ cudaError_t launch_dense_pair(const DenseParams& p, int grid, size_t smem_bytes,
     pdl_attribute(attr[1]);
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, true>, p);
-    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, false>, p);
+    if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, true, false>, p);
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, false, false>, p);
 }
 
 // Largest number of co-resident 2-CTA clusters for the pair kernel (0 on failure).
@@ -679,7 +857,7 @@ int dense_pair_max_clusters(size_t smem_bytes) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, mip_dense_kernel<true, false>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, mip_dense_kernel<true, false, false>, &cfg) != cudaSuccess) {
         (void)cudaGetLastError();
         return 0;
     }

@@ -9,6 +9,7 @@ namespace mip {
 
 constexpr int kBlockM = 128;          // rows of C per CTA (TMEM lanes)
 constexpr int kDenseThreads = 192;    // producer warp, MMA warp, 4 epilogue warps
+constexpr int kGatherThreads = 512;   // the same, two idle warps, and 8 warps that gather operand A from an image
 constexpr int kMaxStages = 12;
 constexpr int kCtrlBytes = 512;       // barriers + TMEM slot + abort word
 constexpr int kStagingBytes = 4 * 2 * 4096;   // epilogue: 4 warps x 2 buffers x (32 rows x 128 B)
@@ -51,11 +52,22 @@ struct alignas(64) DenseParams {
     int a_im2col;
     int conv_wo, conv_howo, conv_s, c_chunks;
     int stride_w, stride_h, pad_w, pad_h, dil_w, dil_h;
+    // software-gathered im2col (operand A built in shared memory by eight extra warps; for images
+    // whose channel count TMA cannot address).  A row of A is R slots of g_slot bytes; slot r is
+    // a copy of the g_slot input bytes that start at the window's first pixel in filter row r
+    // (the first g_seg = S*Cin of them are real taps, the rest meet zero weights).
+    int a_gather;
+    const uint8_t* gx;       // NHWC image batch
+    long long g_xbytes;      // its size (loads never leave [gx, gx + g_xbytes))
+    int g_h, g_row_bytes;    // image rows, bytes per image row (W * Cin)
+    int g_cin, g_seg, g_slot;
+    int g_chunks;            // 16-byte chunks per row of A (R * g_slot / 16)
     unsigned int* status;    // device word, bit 0 set when a bounded wait expired
     unsigned long long wait_budget_ns;
     unsigned long long* trace;   // timeline stamps of CTA 0; only read by builds with -DMIPGEMM_TRACE
 };
 
+cudaError_t launch_dense_gather(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream);
 cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream);
 cudaError_t launch_dense_cluster(const DenseParams& p, int grid, int cluster, size_t smem_bytes, cudaStream_t stream);
 cudaError_t launch_dense_pair(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream);
@@ -95,6 +107,9 @@ cudaError_t launch_repack(const void* src, long long src_pitch, void* dst, long 
                           long long rows, long long cols, cudaStream_t stream);
 cudaError_t launch_transpose_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,
                                     long long rows_out, long long cols_out, cudaStream_t stream);
+// Weights [rows][R][seg] -> [rows][R][slot], zero padded (slot >= seg, slot % 16 == 0).
+cudaError_t launch_weight_slots(const int8_t* src, int8_t* dst, long long rows, int R, int seg, int slot,
+                                cudaStream_t stream);
 cudaError_t launch_fill_zero(int32_t* C, long long ldc, long long M, long long N, cudaStream_t stream);
 struct Im2colParams {
     const uint8_t* X; uint8_t* out;

@@ -42,15 +42,15 @@ def run_gemm(mg, mode, M, N, K, A, B, *, lda=None, ldb=None, C=None, ldc=None, a
     return out, path
 
 
-def run_conv(mg, X, Wt, stride, pad, dil, Y=None, accumulate=False):
+def run_conv(mg, X, Wt, stride, pad, dil, Y=None, accumulate=False, x_misalign=0):
     from oracle.mip_oracle import conv_out_hw
     Nb, H, W, Cin = X.shape
     Cout, R, S, _ = Wt.shape
     Ho, Wo = conv_out_hw(H, W, R, S, stride, pad, dil)
     if Y is None:
         Y = np.full((Nb, Ho, Wo, Cout), 0x7F7F7F7F, dtype=np.int32)
-    dX, _kx = to_dev(X)
-    dW, _kw = to_dev(Wt)
+    dX, _kx = to_dev(X, x_misalign)
+    dW, _kw = to_dev(Wt, x_misalign)
     dY, _ky = to_dev(Y)
     mg.mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride[0], stride[1], pad[0], pad[1],
                             dil[0], dil[1], dX, dW, dY, accumulate)

@@ -78,7 +78,8 @@ def test_workspace_queries(mg):
     qc = mg.mipgemm_workspace_query_conv
     assert qc(32, 56, 56, 64, 64, 3, 3, 1, 1, 1, 1, 1, 1) == 0                  # TMA im2col
     assert qc(32, 56, 56, 64, 256, 1, 1, 1, 1, 0, 0, 1, 1) == 0                 # pointwise
-    assert qc(32, 224, 224, 3, 64, 7, 7, 2, 2, 3, 3, 1, 1) >= 32 * 112 * 112 * 160
+    assert qc(32, 224, 224, 3, 64, 7, 7, 2, 2, 3, 3, 1, 1) == 64 * 7 * 32          # gathered: slot-padded weights only
+    assert qc(2, 32, 32, 3, 64, 3, 3, 1, 1, 2, 2, 2, 2) >= 2 * 32 * 32 * 32        # dilated columns: explicit matrix
 
 
 def test_tuning_validation(mg):

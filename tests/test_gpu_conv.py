@@ -67,11 +67,56 @@ def test_implicit_im2col_tma(mg, case):
                expect_flag=mg.PATH_IM2COL_TMA)
 
 
-EXPLICIT_CASES = [
-    (2, 32, 32, 3, 64, 7, 7, (2, 2), (3, 3), (1, 1)),        # stem-like, Cin = 3, K = 147
-    (2, 12, 12, 16, 32, 3, 3, (1, 1), (1, 1), (1, 1)),       # Cin % 16 == 0 but not % 64
-    (1, 10, 11, 5, 7, 3, 2, (2, 1), (1, 0), (1, 2)),
+GATHER_CASES = [
+    (2, 32, 32, 3, 64, 7, 7, (2, 2), (3, 3), (1, 1)),        # stem-like, Cin = 3, K = 147 (slot 32)
+    (2, 12, 12, 16, 32, 3, 3, (1, 1), (1, 1), (1, 1)),       # Cin % 16 == 0 but not % 64 (slot = segment)
+    (3, 19, 23, 3, 64, 7, 7, (2, 2), (3, 3), (1, 1)),        # odd extents: tiles straddle rows and images
+    (1, 10, 11, 5, 7, 3, 2, (2, 1), (1, 0), (2, 1)),         # dilated rows, Cout % 4 != 0
+    (2, 9, 9, 24, 40, 3, 3, (1, 1), (1, 1), (1, 1)),         # segment 72 -> slot 80, K' = 240 (two k-blocks)
+    (2, 14, 13, 1, 16, 5, 5, (1, 2), (2, 2), (1, 1)),        # one channel
+    (1, 6, 5, 3, 8, 3, 11, (1, 1), (1, 5), (1, 1)),          # filter wider than the image
+    (2, 11, 10, 7, 33, 4, 3, (3, 2), (0, 2), (1, 1)),        # padding only in w, stride 3
+    (1, 40, 40, 100, 48, 3, 3, (1, 1), (1, 1), (1, 1)),      # long rows of A: K' = 912, 8 k-blocks
+    (1, 5, 5, 3, 4, 3, 3, (1, 1), (1, 1), (1, 1)),           # the whole batch is 75 bytes
 ]
+
+
+@pytest.mark.parametrize("case", GATHER_CASES)
+def test_gathered_im2col(mg, case):
+    """Operand A built in shared memory by the gather warps (the augmented matrix never exists)."""
+    Nb, H, W, Cin, Cout, R, S, stride, pad, dil = case
+    check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=20, expect_flag=mg.PATH_IM2COL_GATHER)
+    check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=21, accumulate=True,
+               expect_flag=mg.PATH_IM2COL_GATHER)
+
+
+def test_gathered_im2col_extreme_values(mg):
+    """All taps at their extremes: every sum is the tap count times 255 * -128 (borders have fewer taps)."""
+    Nb, H, W, Cin, Cout, R, S = 2, 17, 15, 3, 16, 7, 7
+    X = np.full((Nb, H, W, Cin), 255, np.uint8)
+    Wt = np.full((Cout, R, S, Cin), -128, np.int8)
+    want = orc.conv(X, Wt, stride=(2, 2), pad=(3, 3))
+    got, path = run_conv(mg, X, Wt, (2, 2), (3, 3), (1, 1))
+    assert path & mg.PATH_IM2COL_GATHER
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("misalign", [1, 2, 3, 7])
+def test_gathered_im2col_any_image_alignment(mg, misalign):
+    Nb, H, W, Cin, Cout, R, S = 2, 21, 18, 3, 24, 7, 7
+    X, Wt = conv_inputs(Nb, H, W, Cin, Cout, R, S, 60 + misalign)
+    want = orc.conv(X, Wt, stride=(2, 2), pad=(3, 3))
+    got, path = run_conv(mg, X, Wt, (2, 2), (3, 3), (1, 1), x_misalign=misalign)
+    assert path & mg.PATH_IM2COL_GATHER
+    assert np.array_equal(got, want), first_mismatch(got, want)
+
+
+EXPLICIT_CASES = [
+    (1, 10, 11, 5, 7, 3, 2, (2, 1), (1, 0), (1, 2)),         # dilated columns: not contiguous in the image
+    (2, 12, 12, 16, 32, 3, 3, (1, 1), (1, 1), (1, 3)),
+    (1, 3, 3, 3, 4, 3, 3, (1, 1), (1, 1), (1, 1)),           # the whole batch is 27 bytes
+]
+FORCED_EXPLICIT_CASES = GATHER_CASES[:3]
 
 
 @pytest.mark.parametrize("case", EXPLICIT_CASES)
@@ -80,6 +125,18 @@ def test_explicit_im2col(mg, case):
     check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=20, expect_flag=mg.PATH_IM2COL_EXPLICIT)
     check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=21, accumulate=True,
                expect_flag=mg.PATH_IM2COL_EXPLICIT)
+
+
+@pytest.mark.parametrize("case", FORCED_EXPLICIT_CASES)
+def test_forced_explicit_im2col(mg, case):
+    Nb, H, W, Cin, Cout, R, S, stride, pad, dil = case
+    mg.mipgemm_set_tuning(force_path=mg.PATH_IM2COL_EXPLICIT)
+    try:
+        check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=22, expect_flag=mg.PATH_IM2COL_EXPLICIT)
+        check_conv(mg, Nb, H, W, Cin, Cout, R, S, stride, pad, dil, seed=23, accumulate=True,
+                   expect_flag=mg.PATH_IM2COL_EXPLICIT)
+    finally:
+        mg.mipgemm_set_tuning()
 
 
 def test_forced_explicit_matches_tma(mg):
