@@ -293,7 +293,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(bar_full + 8u * s, kGather ? 9 : 1);   // + one arrival per gather warp
+            mbar_init(bar_full + 8u * s, kGather ? 1 + 4 * kGatherParities : 1);   // + one arrival per gather warp
             mbar_init(bar_empty + 8u * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -490,32 +490,32 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 }
             }
         }
-    } else if (kGather && warp >= 8) {
-        // ------------------------------------------------------------ software im2col (8 warps)
-        // Thread = every second 16-byte chunk of one row of the tile (one output pixel): warps
-        // 8-11 take the even chunks of rows 0-127, warps 12-15 the odd ones.  For every k-block a
-        // thread writes its (up to) four chunks into the stage in the 128-byte-swizzled K-major
+    } else if (kGather && warp >= kGatherFirstWarp) {
+        // ------------------------------------------------------------ software im2col
+        // Thread = every kGatherParities-th 16-byte chunk of one row of the tile (one output
+        // pixel).  For every k-block a thread writes its chunks into the stage in the 128-byte-swizzled K-major
         // layout the TMA would have produced, makes them visible to the tensor core's proxy and
         // arrives.  The loads of the next k-block (of this or the next tile) are issued before the
         // current one is shifted and stored, so their latency is hidden.  Byte offsets into the
         // batch fit 31 bits (checked by the host).
-        const int row = ((warp - 8) & 3) * 32 + lane;
-        const int parity = (warp - 8) >> 2;
+        const int row = ((warp - kGatherFirstWarp) & 3) * 32 + lane;
+        const int parity = (warp - kGatherFirstWarp) >> 2;
+        constexpr int kCh = 8 / kGatherParities;        // chunks per thread and k-block
         const int xbytes = static_cast<int>(p.g_xbytes);
         const uint32_t align = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(p.gx)) & 3u;
         constexpr int kNone = -0x40000000;
         struct Item {                 // one k-block of one tile, as seen by this thread
-            int src[4], offs[4];      // source byte offset of each chunk (kNone: all zero), offset in its slot
+            int src[kCh], offs[kCh];      // source byte offset of each chunk (kNone: all zero), offset in its slot
             int lo, hi, q0;
-            bool edge;
             uint4 mask;               // slots of 16 or 32 bytes: every chunk of this thread has the same offset
-            uint32_t x[4][5];
+            uint32_t x[kCh][5];
         };
-        const bool fixed_off = p.g_slot <= 32;
+        constexpr int kStride = 16 * kGatherParities;   // bytes of a row of A between two chunks of a thread
+        const bool fixed_off = kStride % p.g_slot == 0;
+        const int r_step = kStride / p.g_slot, off_step = kStride - r_step * p.g_slot;
         // per-tile state of the tile that `prepare` is walking through
         int unit = first_unit, kb = 0, kb_end = 0;
         int h0 = 0, lo = 0, hi = 0, src0 = 0;
-        bool edge = false;
         auto next_item = [&](Item& it) -> bool {     // false: no more work
             while (kb >= kb_end) {
                 if (unit >= total_units) return false;
@@ -536,29 +536,34 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 // the right, the slot's padding bytes are copied as they come (they meet zero weights).
                 lo = max(0, -wb);
                 hi = (p.g_row_bytes - wb >= p.g_seg) ? p.g_slot : p.g_row_bytes - wb;
-                edge = lo > 0 || hi < p.g_slot;
                 src0 = n_img * p.g_h * p.g_row_bytes + wb;
             }
-            it.lo = lo; it.hi = hi; it.edge = edge;
+            it.lo = lo; it.hi = hi;
             it.q0 = kb * 8 + parity;
             int r = (it.q0 * 16) / p.g_slot;
             int off = it.q0 * 16 - r * p.g_slot;
-            it.mask = gather_mask(lo - off, hi - off);
+            it.mask = fixed_off ? gather_mask(lo - off, hi - off) : make_uint4(~0u, ~0u, ~0u, ~0u);
+            // (no branches from here on: the four chunks' dependency chains interleave, which is
+            // what hides the arithmetic latency of a warp that has its scheduler almost to itself)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < kCh; ++c) {
                 const int h = h0 + r * p.dil_h;
-                const bool use = it.q0 + 2 * c < p.g_chunks && off < p.g_seg &&
-                                 static_cast<unsigned>(h) < static_cast<unsigned>(p.g_h) && off < hi && off + 16 > lo;
+                const bool use = (it.q0 + kGatherParities * c < p.g_chunks) & (off < p.g_seg) &
+                                 (static_cast<unsigned>(h) < static_cast<unsigned>(p.g_h)) & (off < hi) &
+                                 (off + 16 > lo);
                 it.src[c] = use ? src0 + h * p.g_row_bytes + off : kNone;
                 it.offs[c] = off;
-                off += 32;
-                while (off >= p.g_slot) { off -= p.g_slot; ++r; }
+                off += off_step;                       // on to the thread's next chunk: r_step slots + off_step bytes
+                r += r_step;
+                const bool wrap = off >= p.g_slot;
+                off -= wrap ? p.g_slot : 0;
+                r += wrap ? 1 : 0;
             }
             // all loads back to back and unconditional (chunks that are all zero, and the few at the
             // very ends of the batch, load the batch's first words instead)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const bool plain = it.src[c] >= 4 && it.src[c] <= xbytes - 24;
+            for (int c = 0; c < kCh; ++c) {
+                const bool plain = (it.src[c] >= 4) & (it.src[c] <= xbytes - 24);
                 const uint32_t* w = reinterpret_cast<const uint32_t*>(
                     (reinterpret_cast<uintptr_t>(p.gx) + static_cast<uintptr_t>(plain ? it.src[c] : 4)) &
                     ~static_cast<uintptr_t>(3));
@@ -575,28 +580,33 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             const bool have_next = next_item(nxt);
             if (!mbar_wait(bar_empty + 8u * s, phase ^ 1u, abort_flag, budget)) break;
             const uint32_t dst = smem_base + s * stage_bytes + static_cast<uint32_t>(row) * 128u;
+            // Chunks past the end of a row of A (last k-block) are stored as well: they meet the
+            // zero fill of B.  Chunks at the very ends of the batch are stored as zero here and
+            // patched below.
+            bool border = false;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                if (cur.q0 + 2 * c < p.g_chunks) {
-                    const uint32_t at = dst + (static_cast<uint32_t>((parity + 2 * c) ^ (row & 7)) << 4);
+            for (int c = 0; c < kCh; ++c) {
+                const int sc = cur.src[c];
+                const bool plain = (sc >= 4) & (sc <= xbytes - 24);
+                border |= (sc != kNone) & !plain;
+                const uint32_t sh = ((static_cast<uint32_t>(sc) + align) & 3u) * 8u;
+                uint4 mk = cur.mask;
+                if (!fixed_off) mk = gather_mask(cur.lo - cur.offs[c], cur.hi - cur.offs[c]);   // (uniform)
+                const uint32_t keep = plain ? ~0u : 0u;
+                uint32_t vv[4];
+                vv[0] = __funnelshift_r(cur.x[c][0], cur.x[c][1], sh) & mk.x & keep;
+                vv[1] = __funnelshift_r(cur.x[c][1], cur.x[c][2], sh) & mk.y & keep;
+                vv[2] = __funnelshift_r(cur.x[c][2], cur.x[c][3], sh) & mk.z & keep;
+                vv[3] = __funnelshift_r(cur.x[c][3], cur.x[c][4], sh) & mk.w & keep;
+                st_shared_v4(dst + (static_cast<uint32_t>((parity + kGatherParities * c) ^ (row & 7)) << 4), vv);
+            }
+            if (border) {
+#pragma unroll
+                for (int c = 0; c < kCh; ++c) {
                     const int sc = cur.src[c];
-                    if (sc != kNone && !(sc >= 4 && sc <= xbytes - 24)) {   // at the very ends of the batch
-                        gather_border_chunk(p.gx, xbytes, sc, cur.lo - cur.offs[c], cur.hi - cur.offs[c], at);
-                    } else {
-                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                        if (sc != kNone) {
-                            const uint32_t sh = ((static_cast<uint32_t>(sc) + align) & 3u) * 8u;
-                            v.x = __funnelshift_r(cur.x[c][0], cur.x[c][1], sh);
-                            v.y = __funnelshift_r(cur.x[c][1], cur.x[c][2], sh);
-                            v.z = __funnelshift_r(cur.x[c][2], cur.x[c][3], sh);
-                            v.w = __funnelshift_r(cur.x[c][3], cur.x[c][4], sh);
-                            uint4 mk = cur.mask;
-                            if (!fixed_off && cur.edge) mk = gather_mask(cur.lo - cur.offs[c], cur.hi - cur.offs[c]);
-                            v.x &= mk.x; v.y &= mk.y; v.z &= mk.z; v.w &= mk.w;
-                        }
-                        uint32_t vv[4] = {v.x, v.y, v.z, v.w};
-                        st_shared_v4(at, vv);
-                    }
+                    if (sc != kNone && !(sc >= 4 && sc <= xbytes - 24))
+                        gather_border_chunk(p.gx, xbytes, sc, cur.lo - cur.offs[c], cur.hi - cur.offs[c],
+                                            dst + (static_cast<uint32_t>((parity + kGatherParities * c) ^ (row & 7)) << 4));
                 }
             }
             fence_proxy_async_smem();

@@ -9,7 +9,11 @@ namespace mip {
 
 constexpr int kBlockM = 128;          // rows of C per CTA (TMEM lanes)
 constexpr int kDenseThreads = 192;    // producer warp, MMA warp, 4 epilogue warps
-constexpr int kGatherThreads = 512;   // the same, two idle warps, and 8 warps that gather operand A from an image
+// Gather form of the dense kernel: 4 * kGatherParities more warps build operand A from an image;
+// warp w of them takes rows 32*(w%4).. of the tile and every kGatherParities-th 16-byte chunk.
+constexpr int kGatherParities = 2;
+constexpr int kGatherFirstWarp = 8;   // (warps 6 and 7 idle: 512 threads)
+constexpr int kGatherThreads = 32 * (kGatherFirstWarp + 4 * kGatherParities);
 constexpr int kMaxStages = 12;
 constexpr int kCtrlBytes = 512;       // barriers + TMEM slot + abort word
 constexpr int kStagingBytes = 4 * 2 * 4096;   // epilogue: 4 warps x 2 buffers x (32 rows x 128 B)
