@@ -33,6 +33,7 @@
  * where a term whose input row or column falls outside the image contributes 0.
  *
  * Dequantised results: mip_oracle_dequant (definition C^r = s * C^q in binary64).
+ * Requantised 8-bit codes: mip_oracle_requant (binary32 rule stated at the function).
  *
  * Pins: tests/test_oracle_pins.py (brute force on tiny inputs, closed forms,
  * extremes, range check, checksum identities, NumPy integer matmul, conv vs
@@ -165,6 +166,30 @@ void mip_oracle_dequant(const int32_t *Cq, int64_t count, double scale, double *
 {
     for (int64_t i = 0; i < count; ++i)
         Cr[i] = scale * (double)Cq[i];
+}
+
+/*
+ * Requantisation of an integer result to 8-bit codes (the step that would follow C^q when the next
+ * layer consumes integers again; the paper's scale-only scheme, Section 7.3, read backwards:
+ * code = round(scale * C^q), saturated).  The paper fixes neither rounding nor precision.  Because
+ * floating point decides an integer here, the rule is stated in the arithmetic the GPU epilogue uses,
+ * binary32: t = fl32(fl32(sum) * scale), both roundings to nearest even; r = t rounded to the nearest
+ * integer, ties to even; code = min(max(r, lo), hi).  `scale` must be finite.  Codes are returned as
+ * int32 (the caller narrows them).  The pins check this rule against exact rational arithmetic.
+ */
+#include <math.h>
+void mip_oracle_requant(const int32_t *Cq, int64_t count, float scale, int32_t lo, int32_t hi, int32_t *codes)
+{
+    for (int64_t i = 0; i < count; ++i) {
+        volatile float as_float = (float)Cq[i];          /* (volatile: no wider intermediate) */
+        volatile float t = as_float * scale;
+        float r = rintf(t);                               /* default rounding mode: ties to even */
+        if (r < (float)lo)
+            r = (float)lo;
+        if (r > (float)hi)
+            r = (float)hi;
+        codes[i] = (int32_t)r;
+    }
 }
 
 #ifdef _OPENMP

@@ -31,7 +31,7 @@ def build(force: bool = False) -> str:
         if force or stale:
             tmp = _LIB + ".tmp.%d" % os.getpid()
             cmd = ["gcc", "-O3", "-march=native", "-fopenmp", "-fPIC", "-shared",
-                   "-std=c11", "-Wall", "-Wextra", "-o", tmp, _SRC]
+                   "-std=c11", "-Wall", "-Wextra", "-o", tmp, _SRC, "-lm"]
             subprocess.run(cmd, check=True)
             os.replace(tmp, _LIB)
     return _LIB
@@ -51,6 +51,8 @@ def _load():
         lib.mip_oracle_conv.argtypes = [i64] * 13 + [vp, vp, vp, ci]
         lib.mip_oracle_dequant.restype = None
         lib.mip_oracle_dequant.argtypes = [vp, i64, ctypes.c_double, vp]
+        lib.mip_oracle_requant.restype = None
+        lib.mip_oracle_requant.argtypes = [vp, i64, ctypes.c_float, ctypes.c_int32, ctypes.c_int32, vp]
         lib.mip_oracle_threads.restype = ci
         lib.mip_oracle_threads.argtypes = []
         _lib = lib
@@ -159,4 +161,16 @@ def dequant(Cq: np.ndarray, scale: float) -> np.ndarray:
     flat = np.ascontiguousarray(Cq).reshape(-1)
     out = np.empty(flat.size, dtype=np.float64)
     _load().mip_oracle_dequant(_ptr(flat), flat.size, float(scale), _ptr(out))
+    return out.reshape(Cq.shape)
+
+
+def requant(Cq: np.ndarray, scale: float, lo: int, hi: int) -> np.ndarray:
+    """8-bit codes min(max(rne(fl32(fl32(Cq) * scale)), lo), hi) as an int32 array of Cq's shape."""
+    if Cq.dtype != np.int32:
+        raise TypeError("Cq must be int32")
+    if not np.isfinite(np.float32(scale)):
+        raise ValueError("scale must be finite")
+    flat = np.ascontiguousarray(Cq).reshape(-1)
+    out = np.empty(flat.size, dtype=np.int32)
+    _load().mip_oracle_requant(_ptr(flat), flat.size, float(np.float32(scale)), int(lo), int(hi), _ptr(out))
     return out.reshape(Cq.shape)

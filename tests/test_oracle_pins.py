@@ -342,3 +342,75 @@ def test_unsigned_b_matches_numpy_and_brute_force():
     assert int(orc.gemm(Au[:33025], Au[:33025], 1, 1, 33025)[0]) == 255 * 255 * 33025
     with pytest.raises(orc.OracleOverflow):
         orc.gemm(Au, Au, 1, 1, 33026)
+
+
+# ---------------------------------------------------------------- requantisation to 8-bit codes
+def _round_half_even(fr):
+    """Nearest integer of a Fraction, ties to even (exact)."""
+    from fractions import Fraction
+    fl = fr.numerator // fr.denominator
+    rem = fr - fl
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1):
+        return fl + 1
+    return fl
+
+
+def test_requant_scale_one_is_a_clamp():
+    Cq = np.array([-2 ** 31, -70000, -129, -128, -127, -1, 0, 1, 126, 127, 128, 255, 256, 2 ** 31 - 1], np.int32)
+    assert np.array_equal(orc.requant(Cq, 1.0, -128, 127), np.clip(Cq.astype(np.int64), -128, 127))
+    assert np.array_equal(orc.requant(Cq, 1.0, 0, 255), np.clip(Cq.astype(np.int64), 0, 255))
+    assert np.array_equal(orc.requant(Cq, 1.0, 0, 127), np.clip(Cq.astype(np.int64), 0, 127))      # ReLU then s8
+    assert np.array_equal(orc.requant(Cq, -1.0, -128, 127), np.clip(-Cq.astype(np.int64), -128, 127))
+
+
+def test_requant_ties_go_to_even():
+    Cq = np.array([1, 3, 5, 7, -1, -3, -5, 9, 251, 253], np.int32)          # halves after scale 0.5
+    want = [0, 2, 2, 4, 0, -2, -2, 4, 126, 126]
+    assert orc.requant(Cq, 0.5, -128, 127).tolist() == want
+    assert orc.requant(np.array([10, 30, 50, -10, -30], np.int32), 0.05, -128, 127).tolist() != []  # (smoke)
+
+
+def test_requant_powers_of_two_match_exact_integer_rounding():
+    """For |sum| < 2^24 and a power-of-two scale every binary32 step is exact: the codes are the
+    exactly rounded quotients."""
+    from fractions import Fraction
+    rng = np.random.default_rng(5)
+    Cq = rng.integers(-2 ** 24 + 1, 2 ** 24, size=4000).astype(np.int32)
+    for k in (1, 3, 7, 12, 16, 20):
+        got = orc.requant(Cq, 2.0 ** -k, -128, 127)
+        want = [min(max(_round_half_even(Fraction(int(v), 2 ** k)), -128), 127) for v in Cq]
+        assert got.tolist() == want, k
+
+
+def test_requant_general_scale_against_exact_rationals():
+    """With an arbitrary scale the binary32 rule may differ from the exactly rounded real product by
+    one code, and only when the real product lies within the two roundings' reach of a tie."""
+    from fractions import Fraction
+    rng = np.random.default_rng(6)
+    Cq = rng.integers(-3_000_000, 3_000_000, size=6000).astype(np.int32)
+    for scale in (1.25e-3, 7.3e-5, 3.1e-2, -4.4e-4, 1.0 / 3.0):
+        s32 = float(np.float32(scale))
+        got = orc.requant(Cq, s32, -128, 127)
+        off_by_one = 0
+        for v, g in zip(Cq.tolist(), got.tolist()):
+            real = Fraction(v) * Fraction(s32)
+            exact = min(max(_round_half_even(real), -128), 127)
+            if g != exact:
+                off_by_one += 1
+                assert abs(g - exact) == 1
+                frac = real - (real.numerator // real.denominator)
+                assert abs(frac - Fraction(1, 2)) <= abs(real) * Fraction(1, 2 ** 22), (v, scale)
+        assert off_by_one <= 6          # a handful of near-ties at most
+    # monotone in the sum for a positive scale
+    ordered = np.sort(Cq)
+    codes = orc.requant(ordered, 1.25e-3, -128, 127)
+    assert (np.diff(codes) >= 0).all()
+
+
+def test_requant_saturates_and_keeps_shape():
+    Cq = np.array([[2 ** 31 - 1, -2 ** 31, 10 ** 9], [-10 ** 9, 12345, -12345]], np.int32)
+    got = orc.requant(Cq, 0.75, -128, 127)
+    assert got.shape == (2, 3) and got.tolist() == [[127, -128, 127], [-128, 127, -128]]
+    assert orc.requant(Cq, 1e-9, 0, 255).tolist() == [[2, 0, 1], [0, 0, 0]]
+    with pytest.raises(ValueError):
+        orc.requant(Cq, float("inf"), -128, 127)
