@@ -111,7 +111,7 @@ def build_layouts(torch, mg, n=8192):
     return probs
 
 
-def build_bert(torch, mg, tokens, dequant=False):
+def build_bert(torch, mg, tokens, dequant=False, requant=False):
     probs = []
     for T in tokens:
         for (name, N, K) in inputs.BERT_GEMMS:
@@ -119,10 +119,14 @@ def build_bert(torch, mg, tokens, dequant=False):
             B = inputs.normal_s8(N * K, inputs.seed_for(4, N + K) + 2, 20.0)
             dA, dB = _dev_bytes(torch, A), _dev_bytes(torch, B)
             dC = torch.empty(T * N, dtype=torch.int32, device="cuda")
-            p = Problem("%s_T%d" % (name, T), "gemm", 2.0 * T * N * K, T * K + N * K + 4.0 * T * N)
+            p = Problem("%s_T%d" % (name, T), "gemm", 2.0 * T * N * K,
+                        T * K + N * K + (1.0 if requant else 4.0) * T * N)
             p.dims = (T, N, K)
             p.bufs = (dA, dB, dC)
-            if dequant:
+            if requant:     # int8 codes written into the front of the same buffer
+                p.calls = [lambda T=T, N=N, K=K, dA=dA, dB=dB, dC=dC:
+                           mg.mipgemm_s8s8s8_requant(T, N, K, dA, K, dB, K, dC, N, 1.25e-3)]
+            elif dequant:
                 p.calls = [lambda T=T, N=N, K=K, dA=dA, dB=dB, dC=dC:
                            mg.mipgemm_s8s8f32_dequant(T, N, K, dA, K, dB, K, dC, N, 1.25e-3)]
             else:
@@ -132,7 +136,7 @@ def build_bert(torch, mg, tokens, dequant=False):
     return probs
 
 
-def build_resnet(torch, mg, batch, dequant=False):
+def build_resnet(torch, mg, batch, dequant=False, requant=False):
     probs = []
     for li, (cnt, H, W, Cin, Cout, R, S, st, pd) in enumerate(inputs.RESNET50_CONVS):
         Ho = (H + 2 * pd - (R - 1) - 1) // st + 1
@@ -143,11 +147,14 @@ def build_resnet(torch, mg, batch, dequant=False):
         dY = torch.empty(batch * Ho * Wo * Cout, dtype=torch.int32, device="cuda")
         M, K = batch * Ho * Wo, R * S * Cin
         p = Problem("conv%02d_%dx%dx%d_%d_%dx%d_s%d" % (li + 1, H, W, Cin, Cout, R, S, st), "conv",
-                    2.0 * M * Cout * K, batch * H * W * Cin + Cout * K + 4.0 * M * Cout)
+                    2.0 * M * Cout * K, batch * H * W * Cin + Cout * K + (1.0 if requant else 4.0) * M * Cout)
         p.dims = (M, Cout, K)
         p.count = cnt
         p.bufs = (dX, dW, dY)
-        if dequant:
+        if requant:         # uint8 codes (ReLU included) written into the front of the same buffer
+            p.calls = [lambda a=(batch, H, W, Cin, Cout, R, S, st, st, pd, pd, 1, 1), dX=dX, dW=dW, dY=dY:
+                       mg.mipgemm_conv_u8s8u8_requant(*a, dX, dW, dY, 7.5e-4)]
+        elif dequant:
             p.calls = [lambda a=(batch, H, W, Cin, Cout, R, S, st, st, pd, pd, 1, 1), dX=dX, dW=dW, dY=dY:
                        mg.mipgemm_conv_u8s8f32_dequant(*a, dX, dW, dY, 7.5e-4)]
         else:
@@ -400,6 +407,8 @@ def main():
     ap.add_argument("--eager", action="store_true", help="plain launches instead of CUDA-graph replay")
     ap.add_argument("--dequant", action="store_true",
                     help="bert/resnet: call the fused-dequantisation entry points (float32 = scale * sum)")
+    ap.add_argument("--requant", action="store_true",
+                    help="bert/resnet: call the requantising entry points (8-bit codes = sat(rne(scale * sum)))")
     ap.add_argument("--only", default="", help="keep only problems whose name contains this text (for profiling)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -431,11 +440,11 @@ def main():
         workload = "square s8*s8->s32 sweep M=N=K in %s, uniform int8, accumulate=0" % sizes
         unit, metric = "TOPS", "int8_gemm_tops"
     elif args.workload == "bert":
-        probs = build_bert(torch, mg, inputs.BERT_TOKENS, args.dequant)
+        probs = build_bert(torch, mg, inputs.BERT_TOKENS, args.dequant, args.requant)
         workload = "BERT base/large encoder GEMMs s8*s8->s32, tokens %s" % inputs.BERT_TOKENS
         unit, metric = "TOPS", "int8_gemm_tops"
     elif args.workload == "resnet":
-        probs = build_resnet(torch, mg, args.batch, args.dequant)
+        probs = build_resnet(torch, mg, args.batch, args.dequant, args.requant)
         workload = "ResNet-50 v1.5 convolutions u8*s8->s32 NHWC, batch %d, 53 layers" % args.batch
         unit, metric = "TOPS", "int8_conv_tops"
     elif args.workload == "attention":
@@ -458,7 +467,9 @@ def main():
             inputs.SKINNY_M, inputs.SKINNY_WEIGHTS)
         unit, metric = "GB/s", "skinny_gemm_gbs"
 
-    if args.dequant and args.workload in ("bert", "resnet"):
+    if args.requant and args.workload in ("bert", "resnet"):
+        workload += ", fused requantisation to 8-bit codes"
+    elif args.dequant and args.workload in ("bert", "resnet"):
         workload += ", fused dequantisation to float32"
     if args.only:
         probs = [p for p in probs if args.only in p.name]

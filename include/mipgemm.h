@@ -130,6 +130,30 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
                          int accumulate, void *stream);
 
 /*
+ * Requantised output: C = sat8(rne(scale * (A * B))), one byte per element (paper Section 7.3 read
+ * backwards: the integer result is scaled back into the 8-bit range so that the next layer can
+ * consume integers again; the paper itself dequantises to FP32 between layers, so this is an
+ * extension of its pipeline).  Rule, in binary32: t = fl32(fl32(sum) * scale), both roundings to
+ * nearest even; r = t rounded to the nearest integer, ties to even; code = min(max(r, lo), hi) with
+ * (lo, hi) = (-128, 127) for int8 codes, (0, 127) with relu != 0, and (0, 255) for uint8 codes (which
+ * therefore include a ReLU).  C then never exists as int32 in memory: a quarter of the bytes.
+ *
+ *   C : device, M x N bytes row-major, ldc >= N counted in bytes, any alignment (16-byte aligned
+ *       base and pitch store fastest).  No accumulate form.  scale must be finite.
+ * Everything else (operands, K limits, errors, stream semantics) as for mipgemm_s8s8s32 /
+ * mipgemm_u8s8s32 / mipgemm_conv_u8s8s32.
+ */
+int mipgemm_s8s8s8_requant(int64_t M, int64_t N, int64_t K,
+                           const int8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                           int8_t *C, int64_t ldc, float scale, int relu, void *stream);
+int mipgemm_u8s8u8_requant(int64_t M, int64_t N, int64_t K,
+                           const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                           uint8_t *C, int64_t ldc, float scale, void *stream);
+int mipgemm_conv_u8s8u8_requant(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int R, int S,
+                                int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                                const uint8_t *X, const int8_t *Wt, uint8_t *Y, float scale, void *stream);
+
+/*
  * General form (paper Section 3, last paragraph: a general GEMM supports transposed inputs and
  * both storage orders for all three operands; the effects on A and B are absorbed below the
  * micro-kernel and a column-major C is handled by swapping the roles of A and B).

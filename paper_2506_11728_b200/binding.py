@@ -43,6 +43,9 @@ SIGNATURES = {
     "mipgemm_s8s8f32_dequant": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]),
     "mipgemm_u8s8f32_dequant": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]),
     "mipgemm_conv_u8s8f32_dequant": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, ctypes.c_float, _vp]),
+    "mipgemm_s8s8s8_requant": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _int, _vp]),
+    "mipgemm_u8s8u8_requant": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]),
+    "mipgemm_conv_u8s8u8_requant": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, ctypes.c_float, _vp]),
     "mipgemm_host_s8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_host_u8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_s8s8s32_static_scratch": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
@@ -136,6 +139,26 @@ def mipgemm_batched_u8s8s32(batch, M, N, K, A, lda, stride_a, B, ldb, stride_b, 
                             accumulate=0, stream=None, check=True) -> int:
     return _check(_lib.mipgemm_batched_u8s8s32(batch, M, N, K, _ptr(A), lda, stride_a, _ptr(B), ldb, stride_b,
                                                _ptr(C), ldc, stride_c, int(bool(accumulate)), _stream(stream)), check)
+
+
+def mipgemm_s8s8s8_requant(M, N, K, A, lda, B, ldb, C, ldc, scale, relu=0, stream=None, check=True) -> int:
+    """C[int8] = sat(rne(scale * (A * B))) (clamped at 0 from below with relu)."""
+    return _check(_lib.mipgemm_s8s8s8_requant(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                              float(scale), int(bool(relu)), _stream(stream)), check)
+
+
+def mipgemm_u8s8u8_requant(M, N, K, A, lda, B, ldb, C, ldc, scale, stream=None, check=True) -> int:
+    """C[uint8] = sat(rne(scale * (A * B))), A unsigned."""
+    return _check(_lib.mipgemm_u8s8u8_requant(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                              float(scale), _stream(stream)), check)
+
+
+def mipgemm_conv_u8s8u8_requant(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w,
+                                X, Wt, Y, scale, stream=None, check=True) -> int:
+    """Y[uint8 NHWC] = sat(rne(scale * Conv(Wt, X)))."""
+    return _check(_lib.mipgemm_conv_u8s8u8_requant(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
+                                                   dil_h, dil_w, _ptr(X), _ptr(Wt), _ptr(Y), float(scale),
+                                                   _stream(stream)), check)
 
 
 def mipgemm_s8s8f32_dequant(M, N, K, A, lda, B, ldb, C, ldc, scale, stream=None, check=True) -> int:

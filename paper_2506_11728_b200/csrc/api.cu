@@ -1,6 +1,7 @@
 // C-ABI entry points of libmipgemm: argument validation, path selection, tensor-map
 // construction, scratch-memory handling and kernel launches.  No arithmetic of the
 // method happens on the host.
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -19,6 +20,8 @@ thread_local int tl_last_cuda_error = 0;
 // Output transform of the call in progress on this thread (set by the *_dequant entry points).
 thread_local int tl_out_f32 = 0;
 thread_local float tl_out_scale = 1.0f;
+// ... or requantisation to 8-bit codes (the *_requant entry points): clamp bounds; C then holds bytes
+thread_local int tl_out_q8 = 0, tl_q_lo = 0, tl_q_hi = 0;
 
 struct Tuning {
     int block_n = 0, stages = 0, split_k = 0, force_path = 0;
@@ -242,7 +245,7 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
     int best_pair = 0, best_bn = 128, best_split = 1;
     double best = 1e30;
     // (an explicit split reduces int32 tiles in global memory, which a float output cannot share)
-    const bool explicit_split = g_tuning.split_k != 0 && !tl_out_f32;
+    const bool explicit_split = g_tuning.split_k != 0 && !tl_out_f32 && !tl_out_q8;
     // (N-contiguous B tiles come in 128-column blocks per CTA: a forced width must respect that)
     const int forced_bn = (g_tuning.block_n && (min_bn <= 64 || g_tuning.block_n == 256)) ? g_tuning.block_n : 0;
     for (int pair = 0; pair <= 1; ++pair) {
@@ -261,7 +264,7 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
             const long long tiles = ((M + rows - 1) / rows) * ((N + bn_use - 1) / bn_use);
             for (int split = 1; split <= 8; split *= 2) {
                 if (split > 1) {
-                    if (pair || explicit_split || g_tuning_no_cluster_split || one_cta_no_split) break;
+                    if (pair || explicit_split || g_tuning_no_cluster_split || one_cta_no_split || tl_out_q8) break;
                     if (tiles * split > sm_count || bn_use / split < 32 || (bn_use / split) % 32 != 0) break;
                     if (pl.k_blocks / split < 2) break;
                 }
@@ -352,6 +355,15 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
     }
     p.out_f32 = tl_out_f32;
     p.out_scale = tl_out_scale;
+    if (tl_out_q8) {   // 8-bit codes: C and ldc address bytes; each thread writes its row's 32 bytes per chunk
+        p.out_q8 = 1;
+        p.q_lo = tl_q_lo;
+        p.q_hi = tl_q_hi;
+        p.c_mode = 4;
+        p.accumulate = 0;
+        p.use_red = 0;
+        p.store_vec = (c_addr % 16 == 0 && ldc % 16 == 0) ? 16 : 1;
+    }
     p.a_im2col = 0;
     p.status = dev->status_word;
     p.wait_budget_ns = 4000000000ull;
@@ -425,13 +437,20 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
         tl_last_path = MIPGEMM_PATH_TRIVIAL | path_flags;
         return MIPGEMM_OK;
     }
-    if (!C || reinterpret_cast<uintptr_t>(C) % 4 != 0) return MIPGEMM_ERR_INVALID_ARG;
+    if (!C || (!tl_out_q8 && reinterpret_cast<uintptr_t>(C) % 4 != 0)) return MIPGEMM_ERR_INVALID_ARG;
     if (K > 0 && (!A || !B)) return MIPGEMM_ERR_INVALID_ARG;
     DeviceState* dev = nullptr;
     int st = get_device(&dev);
     if (st != MIPGEMM_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
 
+    if (K == 0 && tl_out_q8) {   // every sum is 0 and so is its code (q_lo <= 0 <= q_hi)
+        tl_last_path = MIPGEMM_PATH_TRIVIAL | path_flags;
+        cudaError_t e = cudaMemset2DAsync(C, static_cast<size_t>(ldc), 0, static_cast<size_t>(N),
+                                          static_cast<size_t>(M), stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+        return MIPGEMM_OK;
+    }
     if (K == 0) {
         tl_last_path = MIPGEMM_PATH_TRIVIAL | path_flags;
         if (!accumulate) {
@@ -443,7 +462,8 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     }
 
     // ---- skinny path
-    if (M <= 16 && g_tuning.force_path != MIPGEMM_PATH_DENSE && g_tuning.force_path != MIPGEMM_PATH_DENSE_PAIR) {
+    if (M <= 16 && !tl_out_q8 && g_tuning.force_path != MIPGEMM_PATH_DENSE &&
+        g_tuning.force_path != MIPGEMM_PATH_DENSE_PAIR) {
         SkinnyParams sp{A, lda, B, ldb, C, ldc, static_cast<int>(M), static_cast<int>(N),
                         static_cast<int>(K), a_unsigned ? 1 : 0, accumulate ? 1 : 0, tl_out_f32, tl_out_scale};
         if (skinny_ring_supported(sp, dev->sm_count) && !g_tuning_no_skinny_ring) {
@@ -841,7 +861,7 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
         tl_last_path = MIPGEMM_PATH_TRIVIAL;
         return MIPGEMM_OK;
     }
-    if (!X || !Wt || !Y || reinterpret_cast<uintptr_t>(Y) % 4 != 0) return MIPGEMM_ERR_INVALID_ARG;
+    if (!X || !Wt || !Y || (!tl_out_q8 && reinterpret_cast<uintptr_t>(Y) % 4 != 0)) return MIPGEMM_ERR_INVALID_ARG;
 
     if (conv_is_pointwise(g))
         return gemm_impl(true, M, Cout, Cin, X, Cin, Wt, Cin, Y, Cout, accumulate, stream_v, 0);
@@ -1010,6 +1030,36 @@ int mipgemm_conv_u8s8f32_dequant(int64_t Nb, int64_t H, int64_t W, int64_t Cin, 
                                  int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
                                  const uint8_t* X, const int8_t* Wt, float* Y, float scale, void* stream) {
     OutputTransformScope scope(scale);
+    return mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, X, Wt,
+                                reinterpret_cast<int32_t*>(Y), 0, stream);
+}
+
+// Requantisation to 8-bit codes: the integer entry point runs with the epilogue's code transform
+// switched on for this thread; C / Y then address bytes.
+struct RequantScope {
+    RequantScope(float scale, int lo, int hi) { tl_out_q8 = 1; tl_q_lo = lo; tl_q_hi = hi; tl_out_scale = scale; }
+    ~RequantScope() { tl_out_q8 = 0; tl_q_lo = tl_q_hi = 0; tl_out_scale = 1.0f; }
+};
+
+int mipgemm_s8s8s8_requant(int64_t M, int64_t N, int64_t K, const int8_t* A, int64_t lda, const int8_t* B,
+                           int64_t ldb, int8_t* C, int64_t ldc, float scale, int relu, void* stream) {
+    if (!std::isfinite(scale)) return MIPGEMM_ERR_INVALID_ARG;
+    RequantScope scope(scale, relu ? 0 : -128, 127);
+    return gemm_impl(false, M, N, K, A, lda, B, ldb, reinterpret_cast<int32_t*>(C), ldc, 0, stream, 0);
+}
+
+int mipgemm_u8s8u8_requant(int64_t M, int64_t N, int64_t K, const uint8_t* A, int64_t lda, const int8_t* B,
+                           int64_t ldb, uint8_t* C, int64_t ldc, float scale, void* stream) {
+    if (!std::isfinite(scale)) return MIPGEMM_ERR_INVALID_ARG;
+    RequantScope scope(scale, 0, 255);
+    return gemm_impl(true, M, N, K, A, lda, B, ldb, reinterpret_cast<int32_t*>(C), ldc, 0, stream, 0);
+}
+
+int mipgemm_conv_u8s8u8_requant(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int R, int S,
+                                int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                                const uint8_t* X, const int8_t* Wt, uint8_t* Y, float scale, void* stream) {
+    if (!std::isfinite(scale)) return MIPGEMM_ERR_INVALID_ARG;
+    RequantScope scope(scale, 0, 255);
     return mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, X, Wt,
                                 reinterpret_cast<int32_t*>(Y), 0, stream);
 }

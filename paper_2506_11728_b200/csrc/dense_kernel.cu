@@ -73,6 +73,32 @@ __device__ __forceinline__ void dequant_chunk(const DenseParams& p, uint32_t (&v
     for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__int2float_rn(static_cast<int>(v[j])) * p.out_scale);
 }
 
+// Requantised output: the exact int32 sum is converted to binary32 (round to nearest even), multiplied
+// by the scale in binary32, rounded to the nearest integer (ties to even, saturating) and clamped to
+// [q_lo, q_hi]; one byte per element.  `dst` addresses the first of the chunk's `cols` bytes.
+__device__ __forceinline__ void store_q8_chunk(const DenseParams& p, uint8_t* dst, const uint32_t (&v)[32], int cols) {
+    uint32_t w[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        uint32_t packed = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float t = __fmul_rn(__int2float_rn(static_cast<int>(v[4 * g + j])), p.out_scale);
+            const int code = min(max(__float2int_rn(t), p.q_lo), p.q_hi);
+            packed |= (static_cast<uint32_t>(code) & 0xFFu) << (8 * j);
+        }
+        w[g] = packed;
+    }
+    if (cols == 32 && p.store_vec == 16) {
+        st_global_v4(reinterpret_cast<int32_t*>(dst), &w[0]);
+        st_global_v4(reinterpret_cast<int32_t*>(dst + 16), &w[4]);
+        return;
+    }
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+        if (j < cols) dst[j] = static_cast<uint8_t>(w[j >> 2] >> (8 * (j & 3)));
+}
+
 // Writes one 32-column chunk of one row of the tile.
 __device__ __forceinline__ void store_chunk(const DenseParams& p, int32_t* dst, uint32_t (&v)[32], int cols) {
     if (p.use_red) {
@@ -136,19 +162,43 @@ __device__ __forceinline__ void tma_reduce_chunk(const DenseParams& p, uint32_t 
 // `buf` alternates between two buffers; `issuer` is true in exactly one warp.
 __device__ __forceinline__ void tma_store_slab(const DenseParams& p, uint32_t buf, const uint32_t (&v)[32],
                                                int lane, int q, bool issuer, int x, int y, int z = 0) {
+#ifdef MIPGEMM_TRACE
+    const long long ts0 = clock64();
+#endif
     if (issuer && elect_one()) tma_store_wait_read<1>();
+#ifdef MIPGEMM_TRACE
+    const long long ts1 = clock64();
+#endif
     asm volatile("bar.sync 1, 128;" ::: "memory");      // the buffer is free for all four warps
+#ifdef MIPGEMM_TRACE
+    const long long ts2 = clock64();
+#endif
     const int r = q * 32 + lane;
     const uint32_t row = buf + static_cast<uint32_t>(r) * 128u;
 #pragma unroll
     for (int j = 0; j < 8; ++j) st_shared_v4(row + (static_cast<uint32_t>(j ^ (r & 7)) << 4), &v[4 * j]);
+#ifdef MIPGEMM_TRACE
+    const long long ts3 = clock64();
+#endif
     fence_proxy_async_smem();
+#ifdef MIPGEMM_TRACE
+    const long long ts4 = clock64();
+#endif
     asm volatile("bar.sync 1, 128;" ::: "memory");      // all 128 rows are in place
+#ifdef MIPGEMM_TRACE
+    const long long ts5 = clock64();
+#endif
     if (issuer && elect_one()) {
         if (p.batch > 1) tma_store_3d(&p.tmap_c, buf, x, y, z);
         else tma_store_2d(&p.tmap_c, buf, x, y);
         tma_store_commit();
     }
+#ifdef MIPGEMM_TRACE
+    if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) {
+        p.trace[50] += ts1 - ts0; p.trace[51] += ts2 - ts1; p.trace[52] += ts3 - ts2; p.trace[53] += ts4 - ts3;
+        p.trace[54] += ts5 - ts4; p.trace[55] += clock64() - ts5; p.trace[56] += 1;
+    }
+#endif
 }
 
 // Writes one 32 x 32 chunk (thread = row, v = its 32 columns) with fully coalesced 16-byte
@@ -252,7 +302,7 @@ __device__ __noinline__ void gather_border_chunk(const uint8_t* gx, int xbytes, 
     st_shared_v4(smem_dst, w);
 }
 
-template <bool kPair, bool kMN, bool kGather>
+template <bool kPair, bool kMN, bool kGather, bool kQ8>
 __global__ void __launch_bounds__(kGather ? kGatherThreads : kDenseThreads, 1)
 mip_dense_kernel(const __grid_constant__ DenseParams p) {
     constexpr int kGroup = kPair ? 2 : 1;
@@ -623,7 +673,13 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         for (int unit = first_unit; unit < total_units; unit += unit_stride, ++t) {
             const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
             const uint32_t acc = t & 1, acc_phase = (t >> 1) & 1;
+#ifdef MIPGEMM_TRACE
+            const long long tt0 = clock64();
+#endif
             if (!mbar_wait(bar_tfull + 8u * acc, acc_phase, abort_flag, budget)) break;
+#ifdef MIPGEMM_TRACE
+            if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { p.trace[59] += clock64() - tt0; p.trace[60] += 1; }
+#endif
             if (t == 0 && warp == 2) MIP_STAMP(5);
             tc_fence_after();
             const int m_cta = tc.m0 + static_cast<int>(cta_rank) * kBlockM;
@@ -635,6 +691,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             } else if (p.c_mode == 1 || m_cta + q * 32 < p.M) {   // (slab stores need all four warps)
                 const long long c_off = static_cast<long long>(tc.batch) * p.stride_c;
                 int32_t* crow = p.C + c_off + static_cast<long long>(row) * p.ldc + tc.n0;
+                uint8_t* crow8 = kQ8 ? reinterpret_cast<uint8_t*>(p.C) + static_cast<long long>(row) * p.ldc + tc.n0 : nullptr;
                 const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.block_n;
                 const uint32_t my_staging = staging + static_cast<uint32_t>(q) * 8192u;
                 // two register buffers: the TMEM load of the next chunk is in flight while the
@@ -642,9 +699,18 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 uint32_t va[32], vb[32];
                 tmem_ld_32x32(t_row, va);
                 for (int c0 = 0; c0 < n_here; c0 += 64) {
+#ifdef MIPGEMM_TRACE
+                    const long long tw0 = clock64();
+#endif
                     tmem_ld_wait();
+#ifdef MIPGEMM_TRACE
+                    if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { p.trace[57] += clock64() - tw0; p.trace[58] += 1; }
+#endif
                     if (c0 + 32 < n_here) tmem_ld_32x32(t_row + c0 + 32, vb);
                     if (p.out_f32) dequant_chunk(p, va);
+                    if (kQ8 && p.c_mode == 4) {
+                        if (row < p.M) store_q8_chunk(p, crow8 + c0, va, min(32, n_here - c0));
+                    } else
                     if (p.c_mode == 1) tma_store_slab(p, staging, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
                     else if (p.c_mode == 3) coalesced_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
                     else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging, va, lane, tc.n0 + c0, m_cta + q * 32);
@@ -653,6 +719,9 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                         tmem_ld_wait();
                         if (c0 + 64 < n_here) tmem_ld_32x32(t_row + c0 + 64, va);
                         if (p.out_f32) dequant_chunk(p, vb);
+                        if (kQ8 && p.c_mode == 4) {
+                            if (row < p.M) store_q8_chunk(p, crow8 + c0 + 32, vb, min(32, n_here - c0 - 32));
+                        } else
                         if (p.c_mode == 1) tma_store_slab(p, staging + 16384u, vb, lane, q, warp == 2, tc.n0 + c0 + 32, m_cta, tc.batch);
                         else if (p.c_mode == 3) coalesced_chunk(p, my_staging + 4096u, vb, lane, m_cta + q * 32, tc.n0 + c0 + 32, c_off);
                         else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + 4096u, vb, lane, tc.n0 + c0 + 32, m_cta + q * 32);
@@ -761,19 +830,28 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 }
 
 cudaError_t dense_init() {
-    cudaError_t e = cudaFuncSetAttribute(mip_dense_kernel<false, false, false>,
+    cudaError_t e = cudaFuncSetAttribute(mip_dense_kernel<false, false, false, false>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(mip_dense_kernel<false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(mip_dense_kernel<false, true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(mip_dense_kernel<true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(mip_dense_kernel<true, false, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(mip_dense_kernel<true, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(mip_dense_kernel<true, true, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(mip_dense_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(mip_dense_kernel<false, false, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(mip_dense_kernel<false, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(mip_dense_kernel<true, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kSmemBudget);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(mip_dense_kernel<false, false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kSmemBudget);
     return e;
 }
@@ -796,8 +874,10 @@ cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cuda
     cfg.numAttrs = 1;
     // (the M-/N-contiguous operand forms live in an instantiation of their own, so the common
     // kernel's issue loops carry none of their address arithmetic)
-    if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, true, false>, p);
-    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, false>, p);
+    if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, true, false, false>, p);
+    // (so do the 8-bit-code epilogue and the gather form)
+    if (p.out_q8) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, false, true>, p);
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, false, false>, p);
 }
 
 // One CTA per tile with eight additional warps that gather operand A from an image batch.
@@ -811,7 +891,8 @@ cudaError_t launch_dense_gather(const DenseParams& p, int grid, size_t smem_byte
     pdl_attribute(attr[0]);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, true>, p);
+    if (p.out_q8) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, true, true>, p);
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, true, false>, p);
 }
 
 // One-CTA-per-tile kernel launched in clusters of `cluster` CTAs (cluster split-K); `grid` is a
@@ -831,7 +912,7 @@ cudaError_t launch_dense_cluster(const DenseParams& p, int grid, int cluster, si
     pdl_attribute(attr[1]);
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, false>, p);
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, false, false>, p);
 }
 
 // `grid` counts CTAs and must be even: consecutive CTAs form a cluster of two.
@@ -849,8 +930,9 @@ cudaError_t launch_dense_pair(const DenseParams& p, int grid, size_t smem_bytes,
     pdl_attribute(attr[1]);
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, true, false>, p);
-    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, false, false>, p);
+    if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, true, false, false>, p);
+    if (p.out_q8) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, false, false, true>, p);
+    return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, false, false, false>, p);
 }
 
 // Largest number of co-resident 2-CTA clusters for the pair kernel (0 on failure).
@@ -867,7 +949,7 @@ int dense_pair_max_clusters(size_t smem_bytes) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, mip_dense_kernel<true, false, false>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, mip_dense_kernel<true, false, false, false>, &cfg) != cudaSuccess) {
         (void)cudaGetLastError();
         return 0;
     }

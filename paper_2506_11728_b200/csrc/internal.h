@@ -12,7 +12,7 @@ constexpr int kDenseThreads = 192;    // producer warp, MMA warp, 4 epilogue war
 // Gather form of the dense kernel: 4 * kGatherParities more warps build operand A from an image;
 // warp w of them takes rows 32*(w%4).. of the tile and every kGatherParities-th 16-byte chunk.
 constexpr int kGatherParities = 2;
-constexpr int kGatherFirstWarp = 8;   // (warps 6 and 7 idle: 512 threads)
+constexpr int kGatherFirstWarp = 8;
 constexpr int kGatherThreads = 32 * (kGatherFirstWarp + 4 * kGatherParities);
 constexpr int kMaxStages = 12;
 constexpr int kCtrlBytes = 512;       // barriers + TMEM slot + abort word
@@ -47,7 +47,9 @@ struct alignas(64) DenseParams {
     int store_vec;           // 8, 4 or 1 int32 per store instruction
     int out_f32;             // 1: the epilogue writes float32 scale * sum instead of the int32 sum
     float out_scale;
-    int c_mode;              // 0: row-per-thread stores (any alignment), 1: coalesced stores through
+    int out_q8;              // 1: the epilogue writes 8-bit codes min(max(rne(scale * sum), q_lo), q_hi); C and ldc
+    int q_lo, q_hi;          //    then address bytes (c_mode 4)
+    int c_mode;              // 4: 8-bit codes, row-per-thread; 0: row-per-thread stores (any alignment), 1: coalesced stores through
                              // shared memory, 2: TMA tile reduce-add (split-K); 1 and 2 need a 16-byte
                              // aligned C base and ldc % 4 == 0
     uint32_t idesc;          // tcgen05 instruction descriptor
