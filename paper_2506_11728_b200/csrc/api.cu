@@ -252,9 +252,10 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
         if (pair && (dev->pair_clusters <= 0 || one_cta_no_split)) continue;
         if (g_tuning.force_path == MIPGEMM_PATH_DENSE_PAIR && !pair && dev->pair_clusters > 0) continue;
         if (g_tuning.force_path == MIPGEMM_PATH_DENSE && pair) continue;
-        for (int bn = 64; bn <= 256; bn *= 2) {
+        for (int bn = 64; bn <= 256; bn += 32) {      // any multiple of 32 columns is a legal tile width
             int bn_use = bn;
             if (bn < (pair ? min_bn_pair : min_bn)) continue;
+            if (min_bn >= 128 && bn % 128 != 0) continue;   // (N-contiguous B: whole 128-column blocks)
             if (forced_bn) {
                 if (bn != 256) continue;                      // a single candidate: the forced width
                 bn_use = forced_bn;

@@ -73,7 +73,7 @@ def test_ragged_shapes_dense(mg, mode, accumulate):
         mg.mipgemm_set_tuning()
 
 
-@pytest.mark.parametrize("block_n", [64, 128, 256, 96])
+@pytest.mark.parametrize("block_n", [64, 96, 128, 160, 192, 224, 256])
 def test_tile_widths_and_pitches(mg, block_n):
     mg.mipgemm_set_tuning(block_n=block_n)
     try:
@@ -231,7 +231,7 @@ def test_ragged_shapes_cta_pair_kernel(mg, mode, accumulate):
     try:
         for i, (M, N, K) in enumerate(RAGGED + [(513, 300, 272), (1000, 3000, 784)]):
             check_case(mg, mode, M, N, K, accumulate=accumulate, seed=400 + i, expect_path=mg.PATH_DENSE_PAIR)
-        for bn in (64, 128):
+        for bn in (64, 96, 128, 160, 192, 224):      # every tile width the planner may choose
             mg.mipgemm_set_tuning(block_n=bn, force_path=mg.PATH_DENSE_PAIR)
             check_case(mg, mode, 700, 600, 1424, accumulate=accumulate, seed=450 + bn, ldc=604,
                        expect_path=mg.PATH_DENSE_PAIR)
