@@ -407,6 +407,8 @@ def main():
     ap.add_argument("--eager", action="store_true", help="plain launches instead of CUDA-graph replay")
     ap.add_argument("--dequant", action="store_true",
                     help="bert/resnet: call the fused-dequantisation entry points (float32 = scale * sum)")
+    ap.add_argument("--no-weights-hint", action="store_true",
+                    help="skinny: do not declare the weights constant (no early weight fetch across launches)")
     ap.add_argument("--requant", action="store_true",
                     help="bert/resnet: call the requantising entry points (8-bit codes = sat(rne(scale * sum)))")
     ap.add_argument("--only", default="", help="keep only problems whose name contains this text (for profiling)")
@@ -463,8 +465,11 @@ def main():
         unit, metric = "TOPS", "int8_b1_tops"
     else:
         probs = build_skinny(torch, mg)
-        workload = "skinny decode GEMMs s8*s8->s32, M in %s, weights %s, rotated over >=512 MB" % (
-            inputs.SKINNY_M, inputs.SKINNY_WEIGHTS)
+        if not args.no_weights_hint:
+            mg.mipgemm_set_weights_constant(1)      # decode: the weights are never written between calls
+        workload = "skinny decode GEMMs s8*s8->s32, M in %s, weights %s, rotated over >=512 MB%s" % (
+            inputs.SKINNY_M, inputs.SKINNY_WEIGHTS,
+            "" if args.no_weights_hint else ", weights declared constant (mipgemm_set_weights_constant)")
         unit, metric = "GB/s", "skinny_gemm_gbs"
 
     if args.requant and args.workload in ("bert", "resnet"):

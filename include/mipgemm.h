@@ -321,7 +321,18 @@ int mipgemm_version(void);
 int mipgemm_probe_i8_peak(int iters, int *grid_out, double *ops_per_launch,
                           int32_t *sink, void *stream);
 
-/* Overrides for experiments: tile width (0 = heuristic; 64, 128 or 256), pipeline
+/*
+ * A promise about the weights of the skinny-M (GEMV-like, paper Section 7.2 batch-1) calls, process
+ * wide, off by default: with on != 0 the caller guarantees that the B operand of every later call with
+ * M <= 16 is not written by any work still pending on the call's stream when it is enqueued (the
+ * usual case: B holds inference weights).  The streaming kernel then starts fetching B while the
+ * previous kernel on the stream is still draining (programmatic dependent launch); A is read and C is
+ * written only after that kernel has completed, as always.  Results do not change; breaking the
+ * promise reads stale weights.  Returns MIPGEMM_OK.
+ */
+int mipgemm_set_weights_constant(int on);
+
+/* Overrides for experiments: tile width (0 = heuristic; a multiple of 32 up to 256), pipeline
  * depth (0 = heuristic), split-K factor (0 = heuristic, 1 = off), force path. */
 int mipgemm_set_tuning(int block_n, int stages, int split_k, int force_path);
 

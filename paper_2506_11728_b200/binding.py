@@ -60,6 +60,7 @@ SIGNATURES = {
     "mipgemm_version": (_int, []),
     "mipgemm_probe_i8_peak": (_int, [_int, ctypes.POINTER(_int), ctypes.POINTER(ctypes.c_double), _vp, _vp]),
     "mipgemm_set_tuning": (_int, [_int, _int, _int, _int]),
+    "mipgemm_set_weights_constant": (_int, [_int]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
     _fn = getattr(_lib, _name)
@@ -247,6 +248,11 @@ def mipgemm_probe_i8_peak(iters: int, sink, stream=None):
     st = _lib.mipgemm_probe_i8_peak(iters, ctypes.byref(grid), ctypes.byref(ops), _ptr(sink), _stream(stream))
     _check(st, True)
     return grid.value, ops.value
+
+
+def mipgemm_set_weights_constant(on) -> int:
+    """Promise that B of later M <= 16 calls is never written by work still pending on the stream."""
+    return _check(_lib.mipgemm_set_weights_constant(int(bool(on))), True)
 
 
 def mipgemm_set_tuning(block_n=0, stages=0, split_k=0, force_path=0) -> int:

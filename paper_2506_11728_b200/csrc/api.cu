@@ -31,6 +31,7 @@ bool g_tuning_no_cluster_split = false;  // MIPGEMM_NO_CLUSTER_SPLIT=1: split-K 
 bool g_tuning_no_skinny_ring = false;    // MIPGEMM_NO_SKINNY_RING=1: always the register form of the skinny kernel
 bool g_tuning_no_tma_store = false;   // MIPGEMM_DIRECT_STORE=1: force the direct-store epilogue
 std::atomic<uint64_t> g_launches{0};
+std::atomic<int> g_weights_constant{0};  // mipgemm_set_weights_constant
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -483,6 +484,7 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
                 rp.M = static_cast<int>(M); rp.N = static_cast<int>(N); rp.K = static_cast<int>(K);
                 rp.a_unsigned = a_unsigned ? 1 : 0; rp.accumulate = accumulate ? 1 : 0;
                 rp.out_f32 = tl_out_f32; rp.out_scale = tl_out_scale;
+                rp.b_constant = g_weights_constant.load();
                 rp.status = dev->status_word;
                 rp.wait_budget_ns = 4000000000ull;
                 cudaError_t e = launch_skinny_ring(rp, dev->sm_count, stream);
@@ -1117,6 +1119,11 @@ int mipgemm_probe_i8_peak(int iters, int* grid_out, double* ops_per_launch, int3
     if (e != cudaSuccess) return cuda_fail(e);
     if (grid_out) *grid_out = grid;
     if (ops_per_launch) *ops_per_launch = 2.0 * 128 * 256 * 128 * static_cast<double>(iters) * grid;
+    return MIPGEMM_OK;
+}
+
+int mipgemm_set_weights_constant(int on) {
+    g_weights_constant.store(on != 0 ? 1 : 0);
     return MIPGEMM_OK;
 }
 

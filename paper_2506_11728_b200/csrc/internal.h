@@ -100,6 +100,7 @@ struct alignas(64) SkinnyRingParams {
     int M, N, K;
     int a_unsigned, accumulate;
     int out_f32; float out_scale;   // fused dequantisation (see DenseParams)
+    int b_constant;              // 1: B may be fetched before the previous kernel on the stream has completed
     int slots, tokens_in_smem;   // filled in by the launcher
     unsigned int* status;
     unsigned long long wait_budget_ns;

@@ -126,10 +126,12 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
         tma_prefetch_desc(&p.tmap_b);
     }
     // Everything above touched only shared memory and kernel parameters, so it may overlap the
-    // tail of the previous kernel in the stream; nothing below may.
+    // tail of the previous kernel in the stream.  From here on every thread that touches global
+    // memory first waits for that kernel to complete -- except the producer when the caller has
+    // promised constant weights: its loads of B then start while the previous kernel drains.
     pdl_launch_dependents();
-    pdl_wait();
     __syncthreads();
+    if (!(p.b_constant && warp == kRingConsumers)) pdl_wait();
 
     const int units = (p.N + 15) >> 4;
     const int chunks = (p.K + 1023) >> 10;
@@ -257,6 +259,16 @@ cudaError_t launch_ring_t(SkinnyRingParams p, int grid, cudaStream_t stream) {
     p.tokens_in_smem = (kRingSmemMax - fixed - tok_bytes) / kSlotBytes >= 6 ? 1 : 0;
     int slots = (kRingSmemMax - fixed - (p.tokens_in_smem ? tok_bytes : 0)) / kSlotBytes;
     if (slots > kMaxRingSlots) slots = kMaxRingSlots;
+    if (p.b_constant) {
+        // Constant weights: the next call's producer may run while this call still computes, if both
+        // CTAs fit on the SM -- half the shared memory each (still >= 5 slots = 80 KB in flight per CTA).
+        const int half = 112 * 1024;
+        const int fit = (half - fixed - tok_bytes) / kSlotBytes;
+        if (fit >= 5) {
+            p.tokens_in_smem = 1;
+            slots = fit < kMaxRingSlots ? fit : kMaxRingSlots;
+        }
+    }
     p.slots = slots;
     const size_t smem = static_cast<size_t>(slots) * kSlotBytes + fixed + (p.tokens_in_smem ? tok_bytes : 0);
     cudaLaunchConfig_t cfg = {};

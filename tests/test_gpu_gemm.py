@@ -197,6 +197,17 @@ def test_skinny_full_size_weights(mg, NK):
         check_case(mg, "s8", M, N, K, seed=inputs.seed_for(5, M), expect_path=mg.PATH_SKINNY)
 
 
+def test_skinny_with_constant_weights_promise(mg):
+    """The early weight fetch changes no result (several launches back to back on one stream)."""
+    mg.mipgemm_set_weights_constant(1)
+    try:
+        for i, (M, N, K) in enumerate([(1, 4096, 4096), (8, 4096, 1024), (16, 2064, 2048), (4, 11008, 4096)]):
+            check_case(mg, "s8", M, N, K, seed=700 + i, expect_path=mg.PATH_SKINNY)
+            check_case(mg, "u8", M, N, K, seed=710 + i, accumulate=True, expect_path=mg.PATH_SKINNY)
+    finally:
+        mg.mipgemm_set_weights_constant(0)
+
+
 def test_skinny_misaligned_falls_back_to_dense(mg):
     path = check_case(mg, "s8", 4, 300, 100, seed=41)
     assert path & mg.PATH_MASK == mg.PATH_DENSE and path & mg.PATH_REPACK
