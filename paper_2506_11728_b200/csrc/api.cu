@@ -270,7 +270,10 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
                     if (tiles * split > sm_count || bn_use / split < 32 || (bn_use / split) % 32 != 0) break;
                     if (pl.k_blocks / split < 2) break;
                 }
-                const double us = plan_cost_us(pair, bn_use, split, M, N, pl.k_blocks, block_k, dev);
+                double us = plan_cost_us(pair, bn_use, split, M, N, pl.k_blocks, block_k, dev);
+                // widths that are not a power of two re-read A more often (more DRAM traffic and power than
+                // the model sees): they must win by a clear margin
+                if ((bn_use & (bn_use - 1)) != 0) us *= 1.03;
                 if (us < best) {
                     best = us;
                     best_pair = pair;
