@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC_BYTES = {
     "attention": None,
     "paper_b1": None,
-    "square": 1561e6,   # profiles/dense_kernel_square_sweep.md: (6.4 + 8.4 + 55.3 + 606.3 + 7128.4) MB / 5 launches
+    "square": 1936e6,   # profiles/dense_kernel_square_sweep.md, latest capture: (2.2 + 8.5 + 53.2 + 607.9 + 9013.4) MB / 5 launches
     "bert": None,
     "resnet": None,
     "skinny": 58.9e6,   # profiles/skinny_kernel_14336x4096.md: one 14336 x 4096 launch (traffic = algorithmic bytes)
