@@ -106,6 +106,23 @@ def test_unaligned_orders_are_transposed_into_scratch(mg):
     run_ex(mg, 0, 1, 0, 1, 0, 77, 300, 48, pad=(0, 5, 0), seed=82)
 
 
+@pytest.mark.parametrize("ao,bo,ccol", list(itertools.product([0, 1], [0, 1], [0, 1])))
+def test_tiny_and_degenerate_shapes(mg, ao, bo, ccol):
+    for (M, N, K) in [(1, 1, 1), (5, 3, 2), (17, 1, 40), (1, 33, 16), (16, 16, 16), (2, 300, 1)]:
+        run_ex(mg, 1, 1, ao, bo, ccol, M, N, K, seed=100 + M + N + K)
+        run_ex(mg, 0, 0, ao, bo, ccol, M, N, K, accumulate=True, seed=120 + M + N + K)
+    # K == 0: C is zero-filled or left alone; empty problems are no-ops
+    dC, _c = to_dev(np.full(6 * 8, 7, np.int32))
+    mg.mipgemm_gemm_ex(0, 1, ao, bo, ccol, 6, 8, 0, 0, 8, 0, 8, dC, 8, 0)
+    out = dC.cpu().numpy().view(np.int32).reshape(-1, 8)
+    if ccol:        # 8 columns of 6 elements, pitch 8: the two padding elements of each keep their value
+        assert (out[:, :6] == 0).all() and (out[:, 6:] == 7).all()
+    else:
+        assert (out == 0).all()
+    mg.mipgemm_gemm_ex(0, 1, ao, bo, ccol, 0, 8, 5, 0, 8, 0, 8, dC, 8, 0)
+    assert mg.mipgemm_last_path() == mg.PATH_TRIVIAL
+
+
 def test_ex_argument_errors(mg):
     a = b = c = 256
     f = mg.mipgemm_gemm_ex
