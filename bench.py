@@ -631,16 +631,21 @@ def main():
                 mg.mipgemm_host_s8s8s32(n, n, n, hA, n, hB, n, hC, n, 0)
 
         e2e_step()
-        e2e_steps = max(1, min(args.steps, 3))
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for _ in range(e2e_steps):
+        e2e_steps = max(3, min(args.steps, 7))
+        per_step = []
+        for _ in range(e2e_steps):      # (every host call synchronises its stream before it returns)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
             e2e_step()
-        torch.cuda.synchronize()
-        e2e_s = (time.perf_counter() - t0) / e2e_steps
+            torch.cuda.synchronize()
+            per_step.append(time.perf_counter() - t0)
+        # The host link of these boxes is shared with other tenants: single steps stall by 0.2-2 s now and
+        # then (with every build).  The median step is reported; the mean is kept beside it.
+        e2e_s = sorted(per_step)[len(per_step) // 2]
         e2e = {"value": world * step_ops / e2e_s / 1e12, "unit": "TOPS", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "steps": e2e_steps,
-               "api": "mipgemm_host_s8s8s32 (pinned host buffers, cudaMemcpy2DAsync both ways)"}
+               "stat": "median step", "ms_per_step_mean": sum(per_step) / len(per_step) * 1e3,
+               "api": "mipgemm_host_s8s8s32 (pinned host buffers; row blocks pipelined over three streams)"}
         del pinned
 
     # ---- the CPU oracle on a bounded sample of the same workload, same run

@@ -226,7 +226,10 @@ int mipgemm_conv_u8s8f32_dequant(int64_t Nb, int64_t H, int64_t W, int64_t Cin, 
  * memory obtained with cudaMallocAsync on `stream`, runs the device entry point, copies
  * the M x N result back into C (padding columns of the host C are left untouched; with
  * accumulate != 0 the host C is uploaded first), releases the device memory and
- * SYNCHRONISES the stream before returning.  Same return codes as the device variants.
+ * SYNCHRONISES the stream before returning.  Large problems (>= 2048 rows, >= 32 MB) are cut
+ * into row blocks that three streams pipeline -- operands in, compute on `stream`, results
+ * out -- so both directions of the host link are busy at once; pinned host memory is what
+ * makes those copies asynchronous.  Same return codes as the device variants.
  */
 int mipgemm_host_s8s8s32(int64_t M, int64_t N, int64_t K,
                          const int8_t *A, int64_t lda, const int8_t *B, int64_t ldb,

@@ -49,6 +49,7 @@ struct DeviceState {
     int sm_count = 0;
     int pair_clusters = 0;                 // co-resident 2-CTA clusters of the pair kernel
     unsigned int* status_word = nullptr;   // device
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;   // helper streams of the host-buffer entry points
     void* lent = nullptr;
     size_t lent_bytes = 0;
 };
@@ -100,6 +101,10 @@ int get_device(DeviceState** out) {
             if (const char* sr = std::getenv("MIPGEMM_NO_SKINNY_RING")) g_tuning_no_skinny_ring = std::atoi(sr) != 0;
             if ((e = cudaMalloc(&d.status_word, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaMemset(d.status_word, 0, sizeof(unsigned int))) != cudaSuccess) return cuda_fail(e);
+            // (without them the host-buffer entry points simply do not overlap their copies)
+            if (cudaStreamCreateWithFlags(&d.copy_in, cudaStreamNonBlocking) != cudaSuccess) d.copy_in = nullptr;
+            if (cudaStreamCreateWithFlags(&d.copy_out, cudaStreamNonBlocking) != cudaSuccess) d.copy_out = nullptr;
+            (void)cudaGetLastError();
             d.status = MIPGEMM_OK;
         }
         d.ready = true;
@@ -813,10 +818,86 @@ int host_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
         (void)cudaGetLastError();
         return MIPGEMM_ERR_WORKSPACE;
     }
-    void* dA = base;
-    void* dB = base + a_bytes;
+    char* dA = base;
+    char* dB = base + a_bytes;
     int32_t* dC = reinterpret_cast<int32_t*>(base + a_bytes + b_bytes);
     st = MIPGEMM_OK;
+
+    // Large problems are cut into row blocks of A and C, and three streams work on them at once: one
+    // copies operands in, the caller's stream computes, one copies results out, so that the two copy
+    // directions of the link overlap each other and the kernels.
+    const long long total_bytes = static_cast<long long>(M) * K + static_cast<long long>(N) * K +
+                                  4LL * M * N * (accumulate ? 2 : 1);
+    int chunks = 1;
+    if (K > 0 && M >= 2048 && total_bytes >= (32LL << 20) && dev->copy_in && dev->copy_out) {
+        chunks = static_cast<int>(M / 1024);
+        if (chunks > 8) chunks = 8;
+    }
+    if (chunks > 1) {
+        const long long rows_per = round_up((M + chunks - 1) / chunks, 256);
+        chunks = static_cast<int>((M + rows_per - 1) / rows_per);
+        cudaEvent_t ev[4 + 2 * 8];     // start, B, done-in, done-out and two per row block
+        int n_ev = 0;
+        auto new_event = [&](cudaEvent_t* out) -> bool {
+            cudaError_t ee = cudaEventCreateWithFlags(out, cudaEventDisableTiming);
+            if (ee != cudaSuccess) { st = cuda_fail(ee); return false; }
+            ev[n_ev++] = *out;
+            return true;
+        };
+        auto check = [&](cudaError_t ee) -> bool {
+            if (ee != cudaSuccess && st == MIPGEMM_OK) st = cuda_fail(ee);
+            return ee == cudaSuccess;
+        };
+        cudaEvent_t ev_start = nullptr, ev_b = nullptr, ev_done = nullptr;
+        bool ok = new_event(&ev_start) && check(cudaEventRecord(ev_start, stream)) &&
+                  check(cudaStreamWaitEvent(dev->copy_in, ev_start, 0)) &&
+                  check(cudaMemcpy2DAsync(dB, pitch, B, ldb, K, N, cudaMemcpyHostToDevice, dev->copy_in)) &&
+                  new_event(&ev_b) && check(cudaEventRecord(ev_b, dev->copy_in)) &&
+                  check(cudaStreamWaitEvent(stream, ev_b, 0));
+        bool any_out = false;
+        for (int i = 0; i < chunks && ok; ++i) {
+            const long long r0 = i * rows_per;
+            const long long rows = (M - r0 < rows_per) ? M - r0 : rows_per;
+            char* a_i = dA + r0 * pitch;
+            int32_t* c_i = dC + r0 * ldc_dev;
+            cudaEvent_t ev_in = nullptr, ev_cmp = nullptr;
+            ok = check(cudaMemcpy2DAsync(a_i, pitch, static_cast<const char*>(A) + r0 * lda, lda, K, rows,
+                                         cudaMemcpyHostToDevice, dev->copy_in));
+            if (ok && accumulate)
+                ok = check(cudaMemcpy2DAsync(c_i, ldc_dev * 4, C + r0 * ldc, ldc * 4, N * 4, rows,
+                                             cudaMemcpyHostToDevice, dev->copy_in));
+            ok = ok && new_event(&ev_in) && check(cudaEventRecord(ev_in, dev->copy_in)) &&
+                 check(cudaStreamWaitEvent(stream, ev_in, 0));
+            if (ok) {
+                const int gs = gemm_impl(a_unsigned, rows, N, K, a_i, pitch, reinterpret_cast<const int8_t*>(dB), pitch,
+                                         c_i, ldc_dev, accumulate, stream_v, 0);
+                if (gs != MIPGEMM_OK) { st = gs; ok = false; }
+            }
+            ok = ok && new_event(&ev_cmp) && check(cudaEventRecord(ev_cmp, stream)) &&
+                 check(cudaStreamWaitEvent(dev->copy_out, ev_cmp, 0)) &&
+                 check(cudaMemcpy2DAsync(C + r0 * ldc, ldc * 4, c_i, ldc_dev * 4, N * 4, rows, cudaMemcpyDeviceToHost,
+                                         dev->copy_out));
+            any_out = any_out || ok;
+        }
+        // the caller's stream (and the release of the buffer) waits for both helper streams
+        if (new_event(&ev_done)) {
+            if (check(cudaEventRecord(ev_done, dev->copy_in))) check(cudaStreamWaitEvent(stream, ev_done, 0));
+        }
+        cudaEvent_t ev_out = nullptr;
+        if (any_out && new_event(&ev_out)) {
+            if (check(cudaEventRecord(ev_out, dev->copy_out))) check(cudaStreamWaitEvent(stream, ev_out, 0));
+        }
+        (void)cudaFreeAsync(base, stream);
+        e = cudaStreamSynchronize(stream);
+        if (st == MIPGEMM_OK && e != cudaSuccess) st = cuda_fail(e);
+        if (st != MIPGEMM_OK) {   // make sure nothing of this call is still in flight
+            (void)cudaStreamSynchronize(dev->copy_in);
+            (void)cudaStreamSynchronize(dev->copy_out);
+        }
+        for (int i = 0; i < n_ev; ++i) (void)cudaEventDestroy(ev[i]);
+        return st;
+    }
+
     if (K > 0) {
         e = cudaMemcpy2DAsync(dA, pitch, A, lda, K, M, cudaMemcpyHostToDevice, stream);
         if (e == cudaSuccess) e = cudaMemcpy2DAsync(dB, pitch, B, ldb, K, N, cudaMemcpyHostToDevice, stream);
@@ -827,7 +908,7 @@ int host_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
         if (e != cudaSuccess) st = cuda_fail(e);
     }
     if (st == MIPGEMM_OK)
-        st = gemm_impl(a_unsigned, M, N, K, dA, pitch, static_cast<const int8_t*>(dB), pitch, dC, ldc_dev,
+        st = gemm_impl(a_unsigned, M, N, K, dA, pitch, reinterpret_cast<const int8_t*>(dB), pitch, dC, ldc_dev,
                        accumulate, stream_v, 0);
     if (st == MIPGEMM_OK) {
         e = cudaMemcpy2DAsync(C, ldc * 4, dC, ldc_dev * 4, N * 4, M, cudaMemcpyDeviceToHost, stream);
