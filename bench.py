@@ -608,12 +608,8 @@ def main():
                     "traffic": NCU_TRAFFIC_BYTES[args.workload]}
     roofline["launches_timed"] = n_launch
 
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-
-    # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies timed); with several
+    # ranks all of them run it at the same time (they share the host's links) and the slowest rank counts
     e2e = None
     if args.workload == "square" and not args.no_e2e:
         pinned = []
@@ -635,10 +631,13 @@ def main():
         per_step = []
         for _ in range(e2e_steps):      # (every host call synchronises its stream before it returns)
             torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
             t0 = time.perf_counter()
             e2e_step()
             torch.cuda.synchronize()
-            per_step.append(time.perf_counter() - t0)
+            per_step.append(sharding.max_over_ranks(time.perf_counter() - t0, dist if world > 1 else None,
+                                                    torch.device("cuda", local_rank)))
         # The host link of these boxes is shared with other tenants: single steps stall by 0.2-2 s now and
         # then (with every build).  The median step is reported; the mean is kept beside it.
         e2e_s = sorted(per_step)[len(per_step) // 2]
@@ -647,6 +646,11 @@ def main():
                "stat": "median step", "ms_per_step_mean": sum(per_step) / len(per_step) * 1e3,
                "api": "mipgemm_host_s8s8s32 (pinned host buffers; row blocks pipelined over three streams)"}
         del pinned
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # ---- the CPU oracle on a bounded sample of the same workload, same run
     cpu = None
