@@ -545,9 +545,9 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         // Thread = every kGatherParities-th 16-byte chunk of one row of the tile (one output
         // pixel).  For every k-block a thread writes its chunks into the stage in the 128-byte-swizzled K-major
         // layout the TMA would have produced, makes them visible to the tensor core's proxy and
-        // arrives.  The loads of the next k-block (of this or the next tile) are issued before the
-        // current one is shifted and stored, so their latency is hidden.  Byte offsets into the
-        // batch fit 31 bits (checked by the host).
+        // arrives.  (Issuing the next k-block's loads before the current one is stored was measured
+        // and bought nothing: the warps are bound by instruction latency, not by the loads.)  Byte
+        // offsets into the batch fit 31 bits (checked by the host).
         const int row = ((warp - kGatherFirstWarp) & 3) * 32 + lane;
         const int parity = (warp - kGatherFirstWarp) >> 2;
         constexpr int kCh = 8 / kGatherParities;        // chunks per thread and k-block
@@ -566,6 +566,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         // per-tile state of the tile that `prepare` is walking through
         int unit = first_unit, kb = 0, kb_end = 0;
         int h0 = 0, lo = 0, hi = 0, src0 = 0;
+        uint4 tile_mask = make_uint4(~0u, ~0u, ~0u, ~0u);
         auto next_item = [&](Item& it) -> bool {     // false: no more work
             while (kb >= kb_end) {
                 if (unit >= total_units) return false;
@@ -587,12 +588,18 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 lo = max(0, -wb);
                 hi = (p.g_row_bytes - wb >= p.g_seg) ? p.g_slot : p.g_row_bytes - wb;
                 src0 = n_img * p.g_h * p.g_row_bytes + wb;
+                // slots of 16 or 32 bytes: every chunk of this thread sits at the same offset in its slot,
+                // so one mask serves the whole tile
+                if (fixed_off) {
+                    const int off_c = (parity * 16) % p.g_slot;
+                    tile_mask = gather_mask(lo - off_c, hi - off_c);
+                }
             }
             it.lo = lo; it.hi = hi;
             it.q0 = kb * 8 + parity;
             int r = (it.q0 * 16) / p.g_slot;
             int off = it.q0 * 16 - r * p.g_slot;
-            it.mask = fixed_off ? gather_mask(lo - off, hi - off) : make_uint4(~0u, ~0u, ~0u, ~0u);
+            it.mask = tile_mask;
             // (no branches from here on: the four chunks' dependency chains interleave, which is
             // what hides the arithmetic latency of a warp that has its scheduler almost to itself)
 #pragma unroll
@@ -624,10 +631,8 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             return true;
         };
         uint32_t s = 0, phase = 0;
-        Item cur, nxt;
-        bool have = next_item(cur);
-        while (have) {
-            const bool have_next = next_item(nxt);
+        Item cur;
+        while (next_item(cur)) {
             if (!mbar_wait(bar_empty + 8u * s, phase ^ 1u, abort_flag, budget)) break;
             const uint32_t dst = smem_base + s * stage_bytes + static_cast<uint32_t>(row) * 128u;
             // Chunks past the end of a row of A (last k-block) are stored as well: they meet the
@@ -663,8 +668,6 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_full + 8u * s);
             if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
-            cur = nxt;
-            have = have_next;
         }
     } else if (warp < 6) {
         // ------------------------------------------------------------ epilogue
