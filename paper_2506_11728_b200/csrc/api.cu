@@ -589,7 +589,7 @@ bool conv_tma_eligible(const ConvGeom& g, const void* X, const void* Wt) {
 
 // Convolutions TMA cannot gather (channel count not a multiple of 64, e.g. an RGB stem) whose
 // filter rows are contiguous in the image (dil_w == 1): operand A is built in shared memory
-// by eight extra warps of the dense kernel, so the augmented matrix never exists in memory.
+// by extra warps of the dense kernel, so the augmented matrix never exists in memory.
 bool conv_gather_eligible(const ConvGeom& g) {
     if (g.dil_w != 1) return false;
     const long long seg = static_cast<long long>(g.S) * g.Cin;

@@ -883,7 +883,7 @@ cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cuda
     return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, false, false>, p);
 }
 
-// One CTA per tile with eight additional warps that gather operand A from an image batch.
+// One CTA per tile with additional warps (4 * kGatherParities) that gather operand A from an image batch.
 cudaError_t launch_dense_gather(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);

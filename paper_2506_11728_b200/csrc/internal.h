@@ -11,7 +11,7 @@ constexpr int kBlockM = 128;          // rows of C per CTA (TMEM lanes)
 constexpr int kDenseThreads = 192;    // producer warp, MMA warp, 4 epilogue warps
 // Gather form of the dense kernel: 4 * kGatherParities more warps build operand A from an image;
 // warp w of them takes rows 32*(w%4).. of the tile and every kGatherParities-th 16-byte chunk.
-constexpr int kGatherParities = 2;
+constexpr int kGatherParities = 4;
 constexpr int kGatherFirstWarp = 8;
 constexpr int kGatherThreads = 32 * (kGatherFirstWarp + 4 * kGatherParities);
 constexpr int kMaxStages = 12;
@@ -58,7 +58,7 @@ struct alignas(64) DenseParams {
     int a_im2col;
     int conv_wo, conv_howo, conv_s, c_chunks;
     int stride_w, stride_h, pad_w, pad_h, dil_w, dil_h;
-    // software-gathered im2col (operand A built in shared memory by eight extra warps; for images
+    // software-gathered im2col (operand A built in shared memory by extra warps; for images
     // whose channel count TMA cannot address).  A row of A is R slots of g_slot bytes; slot r is
     // a copy of the g_slot input bytes that start at the window's first pixel in filter row r
     // (the first g_seg = S*Cin of them are real taps, the rest meet zero weights).
