@@ -77,17 +77,23 @@ __device__ __forceinline__ void dequant_chunk(const DenseParams& p, uint32_t (&v
 // by the scale in binary32, rounded to the nearest integer (ties to even, saturating) and clamped to
 // [q_lo, q_hi]; one byte per element.  `dst` addresses the first of the chunk's `cols` bytes.
 __device__ __forceinline__ void store_q8_chunk(const DenseParams& p, uint8_t* dst, const uint32_t (&v)[32], int cols) {
+    // The float -> integer step avoids the quarter-rate conversion unit (the epilogue's limit): clamping first
+    // (the bounds are integers, so clamp and round-to-nearest-even commute) leaves |t| < 2^22, where adding
+    // 1.5 * 2^23 rounds t to the nearest integer, ties to even, and leaves its two's complement in the low
+    // mantissa bits.  Same codes as cvt.rni + clamp.
+    const float lo = static_cast<float>(p.q_lo), hi = static_cast<float>(p.q_hi);
     uint32_t w[8];
 #pragma unroll
     for (int g = 0; g < 8; ++g) {
-        uint32_t packed = 0;
+        uint32_t b[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const float t = __fmul_rn(__int2float_rn(static_cast<int>(v[4 * g + j])), p.out_scale);
-            const int code = min(max(__float2int_rn(t), p.q_lo), p.q_hi);
-            packed |= (static_cast<uint32_t>(code) & 0xFFu) << (8 * j);
+            float t = __fmul_rn(__int2float_rn(static_cast<int>(v[4 * g + j])), p.out_scale);
+            t = fminf(fmaxf(t, lo), hi);
+            b[j] = __float_as_uint(__fadd_rn(t, 12582912.0f));
         }
-        w[g] = packed;
+        // byte 0 of b[0..3] -> one word
+        w[g] = __byte_perm(__byte_perm(b[0], b[1], 0x0040), __byte_perm(b[2], b[3], 0x0040), 0x5410);
     }
     if (cols == 32 && p.store_vec == 16) {
         st_global_v4(reinterpret_cast<int32_t*>(dst), &w[0]);
@@ -303,9 +309,12 @@ __device__ __noinline__ void gather_border_chunk(const uint8_t* gx, int xbytes, 
 }
 
 template <bool kPair, bool kMN, bool kGather, bool kQ8>
-__global__ void __launch_bounds__(kGather ? kGatherThreads : kDenseThreads, 1)
+__global__ void __launch_bounds__(kGather ? kGatherThreads : (kQ8 ? kDenseQ8Threads : kDenseThreads), 1)
 mip_dense_kernel(const __grid_constant__ DenseParams p) {
     constexpr int kGroup = kPair ? 2 : 1;
+    // epilogue warps: four (one per quarter of the TMEM lanes); the 8-bit-code epilogue, bound by its
+    // conversion arithmetic, runs eight (two per quarter, alternating 32-column chunks)
+    constexpr int kEpiWarps = (kQ8 && !kGather) ? 8 : 4;
     constexpr int kRowsPerTile = kPair ? 2 * kBlockM : kBlockM;
     const uint32_t cta_rank = kPair ? cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
@@ -348,7 +357,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull + 8u * a, 1);
-            mbar_init(bar_tempty + 8u * a, kPair ? 8 : 4);
+            mbar_init(bar_tempty + 8u * a, kPair ? 2 * kEpiWarps : kEpiWarps);
         }
         mbar_init(bar_drain, 1);
         *abort_flag = 0;
@@ -669,7 +678,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             if (lane == 0) mbar_arrive(bar_full + 8u * s);
             if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
         }
-    } else if (warp < 6) {
+    } else if (warp < 2 + kEpiWarps) {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;
         int t = 0;
@@ -700,6 +709,23 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 // two register buffers: the TMEM load of the next chunk is in flight while the
                 // current one is written out
                 uint32_t va[32], vb[32];
+                if (kQ8 && p.c_mode == 4) {
+                    // 8-bit codes: this warp's chunks are `step` columns apart (the other warp of the
+                    // lane quarter takes the ones in between when there are eight epilogue warps)
+                    constexpr int step = kEpiWarps == 8 ? 64 : 32;
+                    int c0 = kEpiWarps == 8 ? ((warp - 2) >> 2) * 32 : 0;
+                    if (c0 < n_here) tmem_ld_32x32(t_row + c0, va);
+                    for (; c0 < n_here; c0 += 2 * step) {
+                        tmem_ld_wait();
+                        if (c0 + step < n_here) tmem_ld_32x32(t_row + c0 + step, vb);
+                        if (row < p.M) store_q8_chunk(p, crow8 + c0, va, min(32, n_here - c0));
+                        if (c0 + step < n_here) {
+                            tmem_ld_wait();
+                            if (c0 + 2 * step < n_here) tmem_ld_32x32(t_row + c0 + 2 * step, va);
+                            if (row < p.M) store_q8_chunk(p, crow8 + c0 + step, vb, min(32, n_here - c0 - step));
+                        }
+                    }
+                } else {
                 tmem_ld_32x32(t_row, va);
                 for (int c0 = 0; c0 < n_here; c0 += 64) {
 #ifdef MIPGEMM_TRACE
@@ -711,9 +737,6 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 #endif
                     if (c0 + 32 < n_here) tmem_ld_32x32(t_row + c0 + 32, vb);
                     if (p.out_f32) dequant_chunk(p, va);
-                    if (kQ8 && p.c_mode == 4) {
-                        if (row < p.M) store_q8_chunk(p, crow8 + c0, va, min(32, n_here - c0));
-                    } else
                     if (p.c_mode == 1) tma_store_slab(p, staging, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
                     else if (p.c_mode == 3) coalesced_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
                     else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging, va, lane, tc.n0 + c0, m_cta + q * 32);
@@ -722,14 +745,12 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                         tmem_ld_wait();
                         if (c0 + 64 < n_here) tmem_ld_32x32(t_row + c0 + 64, va);
                         if (p.out_f32) dequant_chunk(p, vb);
-                        if (kQ8 && p.c_mode == 4) {
-                            if (row < p.M) store_q8_chunk(p, crow8 + c0 + 32, vb, min(32, n_here - c0 - 32));
-                        } else
                         if (p.c_mode == 1) tma_store_slab(p, staging + 16384u, vb, lane, q, warp == 2, tc.n0 + c0 + 32, m_cta, tc.batch);
                         else if (p.c_mode == 3) coalesced_chunk(p, my_staging + 4096u, vb, lane, m_cta + q * 32, tc.n0 + c0 + 32, c_off);
                         else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + 4096u, vb, lane, tc.n0 + c0 + 32, m_cta + q * 32);
                         else if (row < p.M) store_chunk(p, crow + c0 + 32, vb, min(32, n_here - c0 - 32));
                     }
+                }
                 }
             }
             if (warp == 2) { if (t == 0) MIP_STAMP(6); MIP_STAMP(7); }
@@ -879,7 +900,10 @@ cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cuda
     // kernel's issue loops carry none of their address arithmetic)
     if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, true, false, false>, p);
     // (so do the 8-bit-code epilogue and the gather form)
-    if (p.out_q8) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, false, true>, p);
+    if (p.out_q8) {
+        cfg.blockDim = dim3(kDenseQ8Threads, 1, 1);
+        return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, false, true>, p);
+    }
     return cudaLaunchKernelEx(&cfg, mip_dense_kernel<false, false, false, false>, p);
 }
 
@@ -934,7 +958,10 @@ cudaError_t launch_dense_pair(const DenseParams& p, int grid, size_t smem_bytes,
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     if (p.a_mn || p.b_mn) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, true, false, false>, p);
-    if (p.out_q8) return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, false, false, true>, p);
+    if (p.out_q8) {
+        cfg.blockDim = dim3(kDenseQ8Threads, 1, 1);
+        return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, false, false, true>, p);
+    }
     return cudaLaunchKernelEx(&cfg, mip_dense_kernel<true, false, false, false>, p);
 }
 

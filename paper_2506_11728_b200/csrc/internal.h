@@ -9,6 +9,7 @@ namespace mip {
 
 constexpr int kBlockM = 128;          // rows of C per CTA (TMEM lanes)
 constexpr int kDenseThreads = 192;    // producer warp, MMA warp, 4 epilogue warps
+constexpr int kDenseQ8Threads = 320;  // 8-bit-code epilogue: 8 epilogue warps
 // Gather form of the dense kernel: 4 * kGatherParities more warps build operand A from an image;
 // warp w of them takes rows 32*(w%4).. of the tile and every kGatherParities-th 16-byte chunk.
 constexpr int kGatherParities = 4;
