@@ -725,6 +725,16 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                             if (row < p.M) store_q8_chunk(p, crow8 + c0 + step, vb, min(32, n_here - c0 - step));
                         }
                     }
+                } else if (kGather) {
+                    // (768 threads leave 80 registers per thread: one register buffer, no look-ahead)
+                    for (int c0 = 0; c0 < n_here; c0 += 32) {
+                        tmem_ld_32x32(t_row + c0, va);
+                        tmem_ld_wait();
+                        if (p.out_f32) dequant_chunk(p, va);
+                        if (p.c_mode == 1) tma_store_slab(p, staging + ((c0 >> 5) & 1) * 16384u, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
+                        else if (p.c_mode == 3) coalesced_chunk(p, my_staging + ((c0 >> 5) & 1) * 4096u, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
+                        else if (row < p.M) store_chunk(p, crow + c0, va, min(32, n_here - c0));
+                    }
                 } else {
                 tmem_ld_32x32(t_row, va);
                 for (int c0 = 0; c0 < n_here; c0 += 64) {
