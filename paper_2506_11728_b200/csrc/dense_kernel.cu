@@ -682,6 +682,11 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;
         int t = 0;
+        // Chunks stored so far.  The two staging buffers of the asynchronous store paths alternate with this
+        // running count, not with the chunk's position in its tile: a tile with an odd number of chunks would
+        // otherwise hand the same buffer to two consecutive copies, the second overwriting what the first may
+        // still be reading.
+        uint32_t chunk_no = 0;
         for (int unit = first_unit; unit < total_units; unit += unit_stride, ++t) {
             const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
             const uint32_t acc = t & 1, acc_phase = (t >> 1) & 1;
@@ -731,9 +736,10 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                         tmem_ld_32x32(t_row + c0, va);
                         tmem_ld_wait();
                         if (p.out_f32) dequant_chunk(p, va);
-                        if (p.c_mode == 1) tma_store_slab(p, staging + ((c0 >> 5) & 1) * 16384u, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
-                        else if (p.c_mode == 3) coalesced_chunk(p, my_staging + ((c0 >> 5) & 1) * 4096u, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
+                        if (p.c_mode == 1) tma_store_slab(p, staging + (chunk_no & 1u) * 16384u, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
+                        else if (p.c_mode == 3) coalesced_chunk(p, my_staging + (chunk_no & 1u) * 4096u, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
                         else if (row < p.M) store_chunk(p, crow + c0, va, min(32, n_here - c0));
+                        ++chunk_no;
                     }
                 } else {
                 tmem_ld_32x32(t_row, va);
@@ -747,18 +753,20 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 #endif
                     if (c0 + 32 < n_here) tmem_ld_32x32(t_row + c0 + 32, vb);
                     if (p.out_f32) dequant_chunk(p, va);
-                    if (p.c_mode == 1) tma_store_slab(p, staging, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
+                    if (p.c_mode == 1) tma_store_slab(p, staging + (chunk_no & 1u) * 16384u, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
                     else if (p.c_mode == 3) coalesced_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
-                    else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging, va, lane, tc.n0 + c0, m_cta + q * 32);
+                    else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + (chunk_no & 1u) * 4096u, va, lane, tc.n0 + c0, m_cta + q * 32);
                     else if (row < p.M) store_chunk(p, crow + c0, va, min(32, n_here - c0));
+                    ++chunk_no;
                     if (c0 + 32 < n_here) {
                         tmem_ld_wait();
                         if (c0 + 64 < n_here) tmem_ld_32x32(t_row + c0 + 64, va);
                         if (p.out_f32) dequant_chunk(p, vb);
-                        if (p.c_mode == 1) tma_store_slab(p, staging + 16384u, vb, lane, q, warp == 2, tc.n0 + c0 + 32, m_cta, tc.batch);
+                        if (p.c_mode == 1) tma_store_slab(p, staging + (chunk_no & 1u) * 16384u, vb, lane, q, warp == 2, tc.n0 + c0 + 32, m_cta, tc.batch);
                         else if (p.c_mode == 3) coalesced_chunk(p, my_staging + 4096u, vb, lane, m_cta + q * 32, tc.n0 + c0 + 32, c_off);
-                        else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + 4096u, vb, lane, tc.n0 + c0 + 32, m_cta + q * 32);
+                        else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + (chunk_no & 1u) * 4096u, vb, lane, tc.n0 + c0 + 32, m_cta + q * 32);
                         else if (row < p.M) store_chunk(p, crow + c0 + 32, vb, min(32, n_here - c0 - 32));
+                        ++chunk_no;
                     }
                 }
                 }

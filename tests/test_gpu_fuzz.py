@@ -1,0 +1,157 @@
+"""Seeded random shapes, pitches, alignments and geometries through every entry point, against the oracle.
+MIPGEMM_FUZZ_CASES raises the number of cases per entry point (default 25)."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import mip_oracle as orc
+from paper_2506_11728_b200 import inputs
+from gpu_util import run_gemm, run_conv, to_dev, first_mismatch
+
+pytestmark = pytest.mark.gpu
+CASES = int(os.environ.get("MIPGEMM_FUZZ_CASES", "25"))
+
+
+@pytest.fixture(scope="module")
+def mg():
+    from paper_2506_11728_b200 import binding
+    binding.mipgemm_set_tuning()
+    return binding
+
+
+def dims(rng, big=False):
+    pick = lambda: int(rng.choice([rng.integers(1, 20), rng.integers(20, 200), rng.integers(200, 700 if not big else 1500)]))
+    return pick(), pick(), int(rng.choice([rng.integers(1, 40), rng.integers(40, 300), rng.integers(300, 1200)]))
+
+
+def test_fuzz_gemm(mg):
+    rng = np.random.default_rng(2024)
+    for i in range(CASES):
+        M, N, K = dims(rng, big=True)
+        mode = "u8" if rng.integers(2) else "s8"
+        lda, ldb, ldc = K + int(rng.choice([0, 0, 1, 16, 37])), K + int(rng.choice([0, 0, 3, 16, 48])), N + int(rng.choice([0, 0, 1, 4, 9]))
+        acc = bool(rng.integers(2))
+        A = (inputs.uniform_u8 if mode == "u8" else inputs.uniform_s8)(M * lda, 1000 + i)
+        B = inputs.uniform_s8(N * ldb, 2000 + i)
+        C0 = inputs.uniform_s32(M * ldc, 3000 + i) if acc else None
+        got, path = run_gemm(mg, mode, M, N, K, A, B, lda=lda, ldb=ldb, ldc=ldc, C=None if C0 is None else C0.copy(),
+                             accumulate=acc, misalign_a=int(rng.choice([0, 0, 1, 16])), misalign_b=int(rng.choice([0, 0, 5])))
+        base = C0.copy() if acc else np.full(M * ldc, 0x7F7F7F7F, np.int32)
+        want = orc.gemm(A, B, M, N, K, lda=lda, ldb=ldb, C=base, ldc=ldc, accumulate=acc)
+        assert np.array_equal(got, want), "gemm case %d %s %dx%dx%d ld %d/%d/%d acc %d path %#x: %s" % (
+            i, mode, M, N, K, lda, ldb, ldc, acc, path, first_mismatch(got, want))
+
+
+def test_fuzz_gemm_forced_configurations(mg):
+    """Random tile widths, pipeline depths, split factors and kernel forms (the planner's whole space)."""
+    rng = np.random.default_rng(2028)
+    try:
+        for i in range(CASES):
+            M, N, K = dims(rng, big=True)
+            K = max(K, 16)
+            tune = dict(block_n=int(rng.choice([0, 32, 64, 96, 128, 160, 192, 224, 256])),
+                        stages=int(rng.choice([0, 2, 3, 5])), split_k=int(rng.choice([0, 0, 1, 2, 3, 7])),
+                        force_path=int(rng.choice([0, mg.PATH_DENSE, mg.PATH_DENSE_PAIR])))
+            mg.mipgemm_set_tuning(**tune)
+            mode = "u8" if rng.integers(2) else "s8"
+            acc = bool(rng.integers(2))
+            ldc = N + int(rng.choice([0, 0, 4, 5]))
+            A = (inputs.uniform_u8 if mode == "u8" else inputs.uniform_s8)(M * K, 12000 + i)
+            B = inputs.uniform_s8(N * K, 13000 + i)
+            C0 = inputs.uniform_s32(M * ldc, 14000 + i) if acc else None
+            got, path = run_gemm(mg, mode, M, N, K, A, B, ldc=ldc, C=None if C0 is None else C0.copy(), accumulate=acc)
+            base = C0.copy() if acc else np.full(M * ldc, 0x7F7F7F7F, np.int32)
+            want = orc.gemm(A, B, M, N, K, C=base, ldc=ldc, accumulate=acc)
+            assert np.array_equal(got, want), "forced case %d %s %dx%dx%d ldc %d acc %d %s path %#x: %s" % (
+                i, mode, M, N, K, ldc, acc, tune, path, first_mismatch(got, want))
+    finally:
+        mg.mipgemm_set_tuning()
+
+
+def test_fuzz_gemm_ex(mg):
+    rng = np.random.default_rng(2025)
+    for i in range(CASES):
+        M, N, K = dims(rng)
+        au, bu, ao, bo, cc = (int(rng.integers(2)) for _ in range(5))
+        align = bool(rng.integers(2))
+        if align:       # pitches TMA can address: the operand is read in place
+            M, N, K = (M + 15) // 16 * 16, (N + 15) // 16 * 16, (K + 15) // 16 * 16
+        lda, ldb, ldc = (M if ao else K), (N if bo else K), (M if cc else N) + 4 * int(rng.integers(3))
+        a_rows, b_rows, c_rows = (K if ao else M), (K if bo else N), (N if cc else M)
+        A = (inputs.uniform_u8 if au else inputs.uniform_s8)(a_rows * lda, 4000 + i)
+        B = (inputs.uniform_u8 if bu else inputs.uniform_s8)(b_rows * ldb, 5000 + i)
+        acc = bool(rng.integers(2))
+        C0 = inputs.uniform_s32(c_rows * ldc, 6000 + i)
+        A_can = np.ascontiguousarray(A.reshape(a_rows, lda).T if ao else A.reshape(a_rows, lda))
+        B_can = np.ascontiguousarray(B.reshape(b_rows, ldb).T if bo else B.reshape(b_rows, ldb))
+        C2 = C0.reshape(c_rows, ldc)[:, :(M if cc else N)]
+        C_can = np.ascontiguousarray(C2.T if cc else C2)
+        res = orc.gemm(A_can.reshape(-1), B_can.reshape(-1), M, N, K, C=C_can.reshape(-1).copy(), accumulate=acc).reshape(M, N)
+        want = C0.reshape(c_rows, ldc).copy()
+        want[:, :(M if cc else N)] = res.T if cc else res
+        dA, _a = to_dev(A)
+        dB, _b = to_dev(B)
+        dC, _c = to_dev(C0)
+        mg.mipgemm_gemm_ex(au, bu, ao, bo, cc, M, N, K, dA, lda, dB, ldb, dC, ldc, acc)
+        assert mg.mipgemm_device_status() == mg.OK
+        got = dC.cpu().numpy().view(np.int32).reshape(c_rows, ldc)
+        assert np.array_equal(got, want), "gemm_ex case %d signs %d%d orders %d%d ccol %d %dx%dx%d path %#x" % (
+            i, au, bu, ao, bo, cc, M, N, K, mg.mipgemm_last_path())
+
+
+def test_fuzz_conv(mg):
+    rng = np.random.default_rng(2026)
+    for i in range(CASES):
+        Cin = int(rng.choice([1, 3, 5, 16, 24, 64, 128, 192]))
+        R, S = int(rng.integers(1, 5)), int(rng.integers(1, 5))
+        dil = (int(rng.integers(1, 3)), int(rng.integers(1, 3)))
+        pad = (int(rng.integers(0, 3)), int(rng.integers(0, 3)))
+        stride = (int(rng.integers(1, 4)), int(rng.integers(1, 4)))
+        H = int(rng.integers(dil[0] * (R - 1) + 1, 24)) if dil[0] * (R - 1) + 1 < 24 else dil[0] * (R - 1) + 1
+        W = int(rng.integers(dil[1] * (S - 1) + 1, 24)) if dil[1] * (S - 1) + 1 < 24 else dil[1] * (S - 1) + 1
+        Nb, Cout = int(rng.integers(1, 4)), int(rng.choice([4, 7, 32, 64, 100]))
+        X = inputs.uniform_u8(Nb * H * W * Cin, 7000 + i).reshape(Nb, H, W, Cin)
+        Wt = inputs.normal_s8(Cout * R * S * Cin, 8000 + i, 32.0, -127, 127).reshape(Cout, R, S, Cin)
+        acc = bool(rng.integers(2))
+        Ho, Wo = orc.conv_out_hw(H, W, R, S, stride, pad, dil)
+        Y0 = inputs.uniform_s32(Nb * Ho * Wo * Cout, 9000 + i).reshape(Nb, Ho, Wo, Cout) if acc else None
+        want = orc.conv(X, Wt, stride=stride, pad=pad, dil=dil, Y=None if Y0 is None else Y0.copy(), accumulate=acc)
+        got, path = run_conv(mg, X, Wt, stride, pad, dil, Y=None if Y0 is None else Y0.copy(), accumulate=acc,
+                             x_misalign=int(rng.choice([0, 0, 0, 3])))
+        assert np.array_equal(got, want), "conv case %d %s f%dx%d s%s p%s d%s cout %d acc %d path %#x: %s" % (
+            i, X.shape, R, S, stride, pad, dil, Cout, acc, path, first_mismatch(got, want))
+
+
+def test_fuzz_scaled_outputs(mg):
+    rng = np.random.default_rng(2027)
+    for i in range(CASES):
+        M, N, K = dims(rng)
+        unsigned = bool(rng.integers(2))
+        A = (inputs.uniform_u8 if unsigned else inputs.uniform_s8)(M * K, 10000 + i)
+        B = inputs.uniform_s8(N * K, 11000 + i)
+        sums = orc.gemm(A, B, M, N, K).reshape(M, N)
+        scale = float(np.float32(rng.choice([1.0, 0.5, 2.0 ** -7, 1.3e-3, 7.7e-5]) * (1 if rng.integers(2) else -1)))
+        dA, _a = to_dev(A)
+        dB, _b = to_dev(B)
+        # 8-bit codes
+        ldc = N + int(rng.choice([0, 3, 16]))
+        dC, _c = to_dev(np.full(M * ldc, 0x5A, np.uint8), int(rng.choice([0, 1])))
+        if unsigned:
+            mg.mipgemm_u8s8u8_requant(M, N, K, dA, K, dB, K, dC, ldc, scale)
+            want = orc.requant(sums, scale, 0, 255)
+            got = dC.cpu().numpy().reshape(M, ldc)[:, :N].astype(np.int32)
+        else:
+            relu = int(rng.integers(2))
+            mg.mipgemm_s8s8s8_requant(M, N, K, dA, K, dB, K, dC, ldc, scale, relu)
+            want = orc.requant(sums, scale, 0 if relu else -128, 127)
+            got = dC.cpu().numpy().reshape(M, ldc)[:, :N].view(np.int8).astype(np.int32)
+        assert mg.mipgemm_device_status() == mg.OK
+        assert np.array_equal(got, want), "requant case %d %dx%dx%d scale %g" % (i, M, N, K, scale)
+        assert (dC.cpu().numpy().reshape(M, ldc)[:, N:] == 0x5A).all()
+        # float32
+        dF, _f = to_dev(np.zeros(M * N, np.float32))
+        (mg.mipgemm_u8s8f32_dequant if unsigned else mg.mipgemm_s8s8f32_dequant)(M, N, K, dA, K, dB, K, dF, N, scale)
+        gotf = dF.cpu().numpy().view(np.float32).reshape(M, N)
+        rule = (sums.astype(np.float32) * np.float32(scale)).astype(np.float32)
+        assert np.array_equal(gotf, rule), "dequant case %d" % i

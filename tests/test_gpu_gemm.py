@@ -250,6 +250,22 @@ def test_ragged_shapes_cta_pair_kernel(mg, mode, accumulate):
         mg.mipgemm_set_tuning()
 
 
+def test_odd_chunk_counts_keep_staging_buffers_apart(mg):
+    """Tiles with an odd number of 32-column chunks, many tiles per CTA and almost no main loop: consecutive
+    asynchronous stores (and split-K reduce-adds) must still alternate their staging buffers."""
+    try:
+        for tune, (M, N, K) in [(dict(block_n=96), (150000, 96, 32)), (dict(block_n=32), (100000, 32, 64)),
+                                (dict(block_n=160, force_path=mg.PATH_DENSE_PAIR), (120000, 160, 32)),
+                                (dict(block_n=32, split_k=3, stages=5), (962, 908, 586)),
+                                (dict(block_n=96, split_k=2), (40000, 96, 256))]:
+            mg.mipgemm_set_tuning(**tune)
+            check_case(mg, "s8", M, N, K, seed=900 + N, accumulate=("split_k" in tune))
+        mg.mipgemm_set_tuning()
+        check_case(mg, "u8", 160000, 1000 - 8 * 3, 48, seed=950)          # ragged last tile column: 1 chunk of 8
+    finally:
+        mg.mipgemm_set_tuning()
+
+
 def test_cta_pair_with_unaligned_c_and_repack(mg):
     mg.mipgemm_set_tuning(force_path=mg.PATH_DENSE_PAIR)
     try:
