@@ -69,6 +69,64 @@ def test_fuzz_gemm_forced_configurations(mg):
         mg.mipgemm_set_tuning()
 
 
+def test_fuzz_tall_and_skinny(mg):
+    """Many tiles per CTA with short main loops (tall M, small K), and the M <= 16 streaming kernels."""
+    rng = np.random.default_rng(2029)
+    try:
+        for i in range(CASES):
+            if rng.integers(2):
+                M, N, K = int(rng.integers(20000, 90000)), int(rng.choice([8, 32, 40, 96, 100, 160, 224, 260])), int(rng.choice([16, 32, 64, 80, 128, 200]))
+                mg.mipgemm_set_tuning(block_n=int(rng.choice([0, 0, 32, 96, 160])),
+                                      force_path=int(rng.choice([0, 0, mg.PATH_DENSE, mg.PATH_DENSE_PAIR])))
+            else:
+                M, N, K = int(rng.integers(1, 17)), int(rng.choice([16, 100, 2368, 4096, 5000])), int(rng.choice([128, 256, 1000, 2048, 4096]))
+                mg.mipgemm_set_tuning()
+                mg.mipgemm_set_weights_constant(int(rng.integers(2)))
+            mode = "u8" if rng.integers(2) else "s8"
+            acc = bool(rng.integers(2))
+            A = (inputs.uniform_u8 if mode == "u8" else inputs.uniform_s8)(M * K, 15000 + i)
+            B = inputs.uniform_s8(N * K, 16000 + i)
+            C0 = inputs.uniform_s32(M * N, 17000 + i) if acc else None
+            got, path = run_gemm(mg, mode, M, N, K, A, B, C=None if C0 is None else C0.copy(), accumulate=acc)
+            base = C0.copy() if acc else np.full(M * N, 0x7F7F7F7F, np.int32)
+            want = orc.gemm(A, B, M, N, K, C=base, accumulate=acc)
+            assert np.array_equal(got, want), "tall/skinny case %d %s %dx%dx%d acc %d path %#x: %s" % (
+                i, mode, M, N, K, acc, path, first_mismatch(got, want))
+    finally:
+        mg.mipgemm_set_tuning()
+        mg.mipgemm_set_weights_constant(0)
+
+
+def test_fuzz_batched(mg):
+    rng = np.random.default_rng(2030)
+    for i in range(CASES):
+        batch = int(rng.integers(1, 9))
+        M, N, K = int(rng.integers(1, 300)), int(rng.integers(1, 300)), int(rng.choice([16, 48, 64, 100, 256, 512]))
+        lda, ldb, ldc = K + 16 * int(rng.integers(2)), K + 16 * int(rng.integers(2)), N + 4 * int(rng.integers(3))
+        sa, sb, sc = M * lda + 16 * int(rng.integers(3)), N * ldb, M * ldc + 4 * int(rng.integers(3))
+        acc = bool(rng.integers(2))
+        A = inputs.uniform_s8(batch * sa, 18000 + i)
+        B = inputs.uniform_s8(batch * sb, 19000 + i)
+        C0 = inputs.uniform_s32(batch * sc, 20000 + i)
+        want = C0.copy()
+        for b in range(batch):
+            Cb = np.ascontiguousarray(C0[b * sc:b * sc + M * ldc])
+            res = orc.gemm(A[b * sa:b * sa + M * lda], B[b * sb:b * sb + N * ldb], M, N, K, lda=lda, ldb=ldb, C=Cb.copy(),
+                           ldc=ldc, accumulate=acc)
+            want[b * sc:b * sc + M * ldc] = res
+            if not acc:     # padding columns keep their old value
+                w2 = want[b * sc:b * sc + M * ldc].reshape(M, ldc)
+                w2[:, N:] = C0[b * sc:b * sc + M * ldc].reshape(M, ldc)[:, N:]
+        dA, _a = to_dev(A)
+        dB, _b = to_dev(B)
+        dC, _c = to_dev(C0)
+        mg.mipgemm_batched_s8s8s32(batch, M, N, K, dA, lda, sa, dB, ldb, sb, dC, ldc, sc, acc)
+        assert mg.mipgemm_device_status() == mg.OK
+        got = dC.cpu().numpy().view(np.int32)
+        assert np.array_equal(got, want), "batched case %d b%d %dx%dx%d ld %d/%d/%d acc %d path %#x: %s" % (
+            i, batch, M, N, K, lda, ldb, ldc, acc, mg.mipgemm_last_path(), first_mismatch(got, want))
+
+
 def test_fuzz_gemm_ex(mg):
     rng = np.random.default_rng(2025)
     for i in range(CASES):
@@ -110,7 +168,8 @@ def test_fuzz_conv(mg):
         stride = (int(rng.integers(1, 4)), int(rng.integers(1, 4)))
         H = int(rng.integers(dil[0] * (R - 1) + 1, 24)) if dil[0] * (R - 1) + 1 < 24 else dil[0] * (R - 1) + 1
         W = int(rng.integers(dil[1] * (S - 1) + 1, 24)) if dil[1] * (S - 1) + 1 < 24 else dil[1] * (S - 1) + 1
-        Nb, Cout = int(rng.integers(1, 4)), int(rng.choice([4, 7, 32, 64, 100]))
+        Nb = int(rng.integers(1, 4)) if rng.integers(5) else int(rng.integers(16, 200))     # sometimes many tiles per CTA
+        Cout = int(rng.choice([4, 7, 32, 64, 100]))
         X = inputs.uniform_u8(Nb * H * W * Cin, 7000 + i).reshape(Nb, H, W, Cin)
         Wt = inputs.normal_s8(Cout * R * S * Cin, 8000 + i, 32.0, -127, 127).reshape(Cout, R, S, Cin)
         acc = bool(rng.integers(2))
