@@ -214,3 +214,45 @@ def test_fuzz_scaled_outputs(mg):
         gotf = dF.cpu().numpy().view(np.float32).reshape(M, N)
         rule = (sums.astype(np.float32) * np.float32(scale)).astype(np.float32)
         assert np.array_equal(gotf, rule), "dequant case %d" % i
+
+
+def test_concurrent_callers_on_their_own_streams(mg):
+    """Four host threads, each with its own stream and a mix of paths (dense, skinny, re-pitched, conv, scaled)."""
+    import threading
+    import torch
+    errors = []
+
+    def worker(tid):
+        try:
+            rng = np.random.default_rng(3000 + tid)
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                for i in range(12):
+                    M, N, K = int(rng.choice([5, 300, 1100])), int(rng.integers(40, 600)), int(rng.choice([64, 100, 512, 1000]))
+                    A = inputs.uniform_s8(M * K, 30000 + 100 * tid + i)
+                    B = inputs.uniform_s8(N * K, 31000 + 100 * tid + i)
+                    dA, _a = to_dev(A)
+                    dB, _b = to_dev(B)
+                    dC, _c = to_dev(np.zeros(M * N, np.int32))
+                    sums = orc.gemm(A, B, M, N, K)
+                    if i % 3 == 2:
+                        mg.mipgemm_s8s8f32_dequant(M, N, K, dA, K, dB, K, dC, N, 0.25, stream=stream)
+                        stream.synchronize()
+                        got = dC.cpu().numpy().view(np.float32)
+                        ok = np.array_equal(got, sums.astype(np.float32) * np.float32(0.25))
+                    else:
+                        mg.mipgemm_s8s8s32(M, N, K, dA, K, dB, K, dC, N, 0, stream=stream)
+                        stream.synchronize()
+                        ok = np.array_equal(dC.cpu().numpy().view(np.int32), sums)
+                    if not ok:
+                        errors.append("thread %d case %d %dx%dx%d" % (tid, i, M, N, K))
+        except Exception as exc:      # noqa: BLE001 - reported below
+            errors.append("thread %d: %r" % (tid, exc))
+
+    threads = [threading.Thread(target=worker, args=(t,)) for t in range(4)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    assert mg.mipgemm_device_status() == mg.OK
