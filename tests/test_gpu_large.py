@@ -93,3 +93,23 @@ def test_bert_shapes_large_t_sampled(mg, T):
         C, _ = run_gemm(mg, "s8", T, N, K, A, B)
         sampled_parity(A, B, C, T, N, K, rng, n_rows=16, n_tiles=8)
         checksum_identities(A, B, C, T, N, K, rng)
+
+
+@pytest.mark.parametrize("M,N,K,accumulate", [(3_000_000, 1024, 32, False), (2_500_000, 1100, 48, True)])
+def test_more_than_2_to_31_elements_of_c(mg, M, N, K, accumulate):
+    """C with more than 2^31 elements (12 GB): every address computation must be 64-bit.  Rows around the
+    2^31- and 2^32-element marks, the first and last rows and 300 random rows are checked against the oracle."""
+    import torch
+    A = inputs.uniform_s8(M * K, 41)
+    B = inputs.uniform_s8(N * K, 42)
+    dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    dC = torch.full((M * N,), 7, dtype=torch.int32, device="cuda")
+    mg.mipgemm_s8s8s32(M, N, K, dA, K, dB, K, dC, N, accumulate)
+    assert mg.mipgemm_device_status() == mg.OK
+    marks = np.array([2 ** 31 // N - 1, 2 ** 31 // N, 2 ** 31 // N + 1, 2 ** 32 // N, 2 ** 32 // N + 1]) % M
+    rows = np.unique(np.concatenate([np.arange(0, 4), np.arange(M - 4, M), marks,
+                                     np.random.default_rng(0).integers(0, M, 300)]))
+    got = dC.view(M, N)[torch.from_numpy(rows).cuda()].cpu().numpy()
+    want = orc.gemm(np.ascontiguousarray(A.reshape(M, K)[rows]).reshape(-1), B, len(rows), N, K,
+                    C=np.full(len(rows) * N, 7, np.int32), accumulate=accumulate).reshape(len(rows), N)
+    assert np.array_equal(got, want)
