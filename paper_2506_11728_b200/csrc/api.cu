@@ -363,6 +363,9 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
             p.c_mode = (accumulate || !tma_ok) ? 3 : 1;
         }
     }
+    // A C that is only 4-byte aligned: rows through shared memory, one 128-byte run per store instruction
+    // (split-K partial sums keep the scalar reduce-add form).
+    if (p.c_mode == 0 && !p.use_red && !g_tuning_no_tma_store) p.c_mode = 5;
     p.out_f32 = tl_out_f32;
     p.out_scale = tl_out_scale;
     if (tl_out_q8) {   // 8-bit codes: C and ldc address bytes; each thread writes its row's 32 bytes per chunk
@@ -758,8 +761,8 @@ int batched_impl(bool a_unsigned, int64_t batch, int64_t M, int64_t N, int64_t K
     fill_common(p, pl, M, N, C, ldc, block_k, a_unsigned, accumulate, dev);
     p.batch = static_cast<int>(batch);
     p.stride_c = stride_c;
-    if (stride_c % 4 != 0 && p.c_mode != 0) {   // batch members of C would lose their 16-byte alignment
-        p.c_mode = 0;
+    if (stride_c % 4 != 0 && (p.c_mode == 1 || p.c_mode == 3)) {   // batch members of C would lose their 16-byte alignment
+        p.c_mode = 5;
     }
     auto encode3 = [&](CUtensorMap* map, const void* base, long long inner, long long rows, long long pitch,
                        long long bstride, int box_inner, int box_rows, CUtensorMapDataType dt, int esize) -> int {

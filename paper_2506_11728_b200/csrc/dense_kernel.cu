@@ -308,6 +308,48 @@ __device__ __noinline__ void gather_border_chunk(const uint8_t* gx, int xbytes, 
     st_shared_v4(smem_dst, w);
 }
 
+// Same idea for a C that is only 4-byte aligned (odd pitch or base): the chunk goes through the warp's
+// staging buffer and is written one row per instruction, lane = column, so that every access of the
+// warp is one contiguous 128-byte run instead of 32 words 4*ldc bytes apart.  With accumulate the
+// incoming C is read the same way.  Warp-collective.
+__device__ __forceinline__ void rows_chunk(const DenseParams& p, uint32_t buf, const uint32_t (&v)[32], int lane,
+                                           int row0, int col0, long long c_off) {
+    __syncwarp();   // the previous chunk's reads of `buf` are done
+    const uint32_t mine = buf + static_cast<uint32_t>(lane) * 128u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) st_shared_v4(mine + (static_cast<uint32_t>(j ^ (lane & 7)) << 4), &v[4 * j]);
+    __syncwarp();
+    const int col = col0 + lane;
+    if (col >= p.N) return;
+    int32_t* dst = p.C + c_off + static_cast<long long>(row0) * p.ldc + col;
+    const int rows = min(32, p.M - row0);
+    if (!p.accumulate) {
+        for (int r = 0; r < rows; ++r) {
+            uint32_t x;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(x)
+                         : "r"(buf + static_cast<uint32_t>(r) * 128u + (static_cast<uint32_t>((lane >> 2) ^ (r & 7)) << 4) +
+                               static_cast<uint32_t>(lane & 3) * 4u) : "memory");
+            *dst = static_cast<int32_t>(x);
+            dst += p.ldc;
+        }
+        return;
+    }
+    // all loads of the incoming C first: 32 independent accesses in flight instead of 32 round trips
+    uint32_t c[32];
+#pragma unroll
+    for (int r = 0; r < 32; ++r) c[r] = r < rows ? static_cast<uint32_t>(dst[static_cast<long long>(r) * p.ldc]) : 0u;
+#pragma unroll
+    for (int r = 0; r < 32; ++r) {
+        if (r < rows) {
+            uint32_t x;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(x)
+                         : "r"(buf + static_cast<uint32_t>(r) * 128u + (static_cast<uint32_t>((lane >> 2) ^ (r & 7)) << 4) +
+                               static_cast<uint32_t>(lane & 3) * 4u) : "memory");
+            dst[static_cast<long long>(r) * p.ldc] = static_cast<int32_t>(x + c[r]);
+        }
+    }
+}
+
 template <bool kPair, bool kMN, bool kGather, bool kQ8>
 __global__ void __launch_bounds__(kGather ? kGatherThreads : (kQ8 ? kDenseQ8Threads : kDenseThreads), 1)
 mip_dense_kernel(const __grid_constant__ DenseParams p) {
@@ -738,6 +780,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                         if (p.out_f32) dequant_chunk(p, va);
                         if (p.c_mode == 1) tma_store_slab(p, staging + (chunk_no & 1u) * 16384u, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
                         else if (p.c_mode == 3) coalesced_chunk(p, my_staging + (chunk_no & 1u) * 4096u, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
+                        else if (p.c_mode == 5) rows_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
                         else if (row < p.M) store_chunk(p, crow + c0, va, min(32, n_here - c0));
                         ++chunk_no;
                     }
@@ -756,6 +799,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     if (p.c_mode == 1) tma_store_slab(p, staging + (chunk_no & 1u) * 16384u, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
                     else if (p.c_mode == 3) coalesced_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
                     else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + (chunk_no & 1u) * 4096u, va, lane, tc.n0 + c0, m_cta + q * 32);
+                    else if (p.c_mode == 5) rows_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
                     else if (row < p.M) store_chunk(p, crow + c0, va, min(32, n_here - c0));
                     ++chunk_no;
                     if (c0 + 32 < n_here) {
@@ -765,6 +809,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                         if (p.c_mode == 1) tma_store_slab(p, staging + (chunk_no & 1u) * 16384u, vb, lane, q, warp == 2, tc.n0 + c0 + 32, m_cta, tc.batch);
                         else if (p.c_mode == 3) coalesced_chunk(p, my_staging + 4096u, vb, lane, m_cta + q * 32, tc.n0 + c0 + 32, c_off);
                         else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + (chunk_no & 1u) * 4096u, vb, lane, tc.n0 + c0 + 32, m_cta + q * 32);
+                        else if (p.c_mode == 5) rows_chunk(p, my_staging + 4096u, vb, lane, m_cta + q * 32, tc.n0 + c0 + 32, c_off);
                         else if (row < p.M) store_chunk(p, crow + c0 + 32, vb, min(32, n_here - c0 - 32));
                         ++chunk_no;
                     }

@@ -50,7 +50,8 @@ struct alignas(64) DenseParams {
     float out_scale;
     int out_q8;              // 1: the epilogue writes 8-bit codes min(max(rne(scale * sum), q_lo), q_hi); C and ldc
     int q_lo, q_hi;          //    then address bytes (c_mode 4)
-    int c_mode;              // 4: 8-bit codes, row-per-thread; 0: row-per-thread stores (any alignment), 1: coalesced stores through
+    int c_mode;              // 5: rows through shared memory, 4-byte accesses (C only 4-byte aligned); 4: 8-bit codes,
+                             // row-per-thread; 0: row-per-thread stores (any alignment), 1: coalesced stores through
                              // shared memory, 2: TMA tile reduce-add (split-K); 1 and 2 need a 16-byte
                              // aligned C base and ldc % 4 == 0
     uint32_t idesc;          // tcgen05 instruction descriptor
