@@ -256,3 +256,38 @@ def test_concurrent_callers_on_their_own_streams(mg):
         t.join()
     assert not errors, errors
     assert mg.mipgemm_device_status() == mg.OK
+
+
+def test_fuzz_host_entry_and_lent_workspace(mg):
+    """Host-buffer calls (single block and pipelined row blocks) and device calls with a lent workspace."""
+    import torch
+    rng = np.random.default_rng(2031)
+    ws = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+    try:
+        for i in range(max(6, CASES // 3)):
+            big = bool(rng.integers(2))
+            M = int(rng.integers(2048, 6000)) if big else int(rng.integers(1, 900))
+            N = int(rng.integers(1500, 2600)) if big else int(rng.integers(1, 500))
+            K = int(rng.choice([512, 1000, 2048])) if big else int(rng.integers(1, 700))
+            mode = "u8" if rng.integers(2) else "s8"
+            acc = bool(rng.integers(2))
+            lda, ldb, ldc = K + int(rng.choice([0, 5, 16])), K + int(rng.choice([0, 3])), N + int(rng.choice([0, 1, 8]))
+            A = (inputs.uniform_u8 if mode == "u8" else inputs.uniform_s8)(M * lda, 21000 + i)
+            B = inputs.uniform_s8(N * ldb, 22000 + i)
+            C0 = inputs.uniform_s32(M * ldc, 23000 + i)
+            rows = np.arange(M) if not big else np.unique(np.concatenate([np.arange(3), np.arange(M - 3, M), rng.integers(0, M, 24)]))
+            want = orc.gemm(np.ascontiguousarray(A.reshape(M, lda)[rows]).reshape(-1), B, len(rows), N, K, lda=lda, ldb=ldb,
+                            C=np.ascontiguousarray(C0.reshape(M, ldc)[rows]).reshape(-1), ldc=ldc, accumulate=acc)
+            # host entry
+            hA, hB, hC = torch.from_numpy(A.copy()), torch.from_numpy(B.copy()), torch.from_numpy(C0.copy())
+            if rng.integers(2):
+                hA, hB, hC = hA.pin_memory(), hB.pin_memory(), hC.pin_memory()
+            (mg.mipgemm_host_u8s8s32 if mode == "u8" else mg.mipgemm_host_s8s8s32)(M, N, K, hA, lda, hB, ldb, hC, ldc, acc)
+            assert np.array_equal(hC.numpy().reshape(M, ldc)[rows].reshape(-1), want), "host case %d %dx%dx%d" % (i, M, N, K)
+            # device entry with a lent workspace (re-pitching scratch comes out of it)
+            mg.mipgemm_set_workspace(ws, ws.numel())
+            got, path = run_gemm(mg, mode, M, N, K, A, B, lda=lda, ldb=ldb, ldc=ldc, C=C0.copy(), accumulate=acc)
+            mg.mipgemm_set_workspace(None, 0)
+            assert np.array_equal(got.reshape(M, ldc)[rows].reshape(-1), want), "lent case %d %dx%dx%d path %#x" % (i, M, N, K, path)
+    finally:
+        mg.mipgemm_set_workspace(None, 0)
