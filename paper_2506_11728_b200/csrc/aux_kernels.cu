@@ -111,7 +111,7 @@ cudaError_t launch_weight_slots(const int8_t* src, int8_t* dst, long long rows, 
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_allowed();
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, mip_weight_slots_kernel, src, dst, total, R, seg, slot);

@@ -946,7 +946,7 @@ cudaError_t dense_init() {
 // All launches allow programmatic stream serialisation (see pdl_wait() in the kernel).
 static void pdl_attribute(cudaLaunchAttribute& a) {
     a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    a.val.programmaticStreamSerializationAllowed = 1;
+    a.val.programmaticStreamSerializationAllowed = pdl_allowed();
 }
 
 cudaError_t launch_dense(const DenseParams& p, int grid, size_t smem_bytes, cudaStream_t stream) {

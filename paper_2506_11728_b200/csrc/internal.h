@@ -2,10 +2,18 @@
 #pragma once
 #include <cstddef>
 #include <cstdint>
+#include <cstdlib>
 #include <cuda.h>
 #include <cuda_runtime.h>
 
 namespace mip {
+
+// Programmatic dependent launch may be switched off for experiments (MIPGEMM_NO_PDL=1): every launch then
+// waits for its predecessor in the stream to complete before any of its blocks starts.
+inline int pdl_allowed() {
+    static const int v = [] { const char* e = std::getenv("MIPGEMM_NO_PDL"); return (e && std::atoi(e)) ? 0 : 1; }();
+    return v;
+}
 
 constexpr int kBlockM = 128;          // rows of C per CTA (TMEM lanes)
 constexpr int kDenseThreads = 192;    // producer warp, MMA warp, 4 epilogue warps
@@ -102,6 +110,7 @@ struct alignas(64) SkinnyRingParams {
     int M, N, K;
     int a_unsigned, accumulate;
     int out_f32; float out_scale;   // fused dequantisation (see DenseParams)
+    int pdl_mode;                // 1: launched with programmatic stream serialisation (filled in by the launcher)
     int b_constant;              // 1: B may be fetched before the previous kernel on the stream has completed
     int slots, tokens_in_smem;   // filled in by the launcher
     unsigned int* status;

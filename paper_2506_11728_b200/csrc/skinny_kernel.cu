@@ -112,8 +112,8 @@ mip_skinny_kernel(const SkinnyParams p, int split) {
     constexpr int kDepth = MIP_SKINNY_DEPTH;   // slices in flight per warp
     __shared__ int red[kSkinnyWarps][16][17];        // per-warp partials [weight row][token]
     __shared__ int gather[kSkinnyMaxSplit][256];     // rank 0 only: per-CTA partials of the cluster
-    pdl_launch_dependents();   // (programmatic dependent launch: see ptx.cuh)
-    pdl_wait();
+    pdl_wait();                // (programmatic dependent launch: see ptx.cuh)
+    pdl_launch_dependents();   // released only now: at most two kernels of a chain are in flight
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
     const uint32_t rank = split > 1 ? cluster_ctarank() : 0u;
@@ -226,8 +226,10 @@ static cudaError_t launch_skinny_t(const SkinnyParams& p, int split, cudaStream_
     attr[0].val.clusterDim.x = static_cast<unsigned>(split);
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // (measured: these many-CTA streaming kernels gain nothing from an early launch of their successor and
+    // lose 3-4 % in CUDA-graph chains, so the attribute stays off; the in-kernel instructions are then no-ops)
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].val.programmaticStreamSerializationAllowed = 0;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, mip_skinny_kernel<kU, kTwo>, p, split);
