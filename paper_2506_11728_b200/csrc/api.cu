@@ -215,8 +215,8 @@ struct Plan {
 // Cost model behind the plan (clocks, calibrated on B200 with CUDA-graph timings of this
 // kernel).  One 128-byte k-block of a 128 x bn tile costs what the slower of the tensor pipe
 // (2*bn clk) and the SM's ~64 B/clk ingest from L2 allows; CTA pairs stage only half of B per
-// CTA.  The epilogue of a tile (350 clk per 32-column chunk) hides behind the next tile's main
-// loop; only the last one is exposed.  A launch carries ~3.7 us of fixed cost (launch gap,
+// CTA.  The epilogue of a tile hides behind the next tile's main loop as far as the store pace
+// allows (see below); the last one (350 clk per 32-column chunk) is exposed.  A launch carries ~3.7 us of fixed cost (launch gap,
 // set-up, pipeline fill, store drain); the DSMEM exchange of a cluster split-K costs about
 // 2.5 / 6 / 13 us for 2 / 4 / 8 CTAs (measured), so it only pays for K-heavy, tile-poor shapes.
 double plan_cost_us(int pair, int bn, int split, long long M, long long N, int k_blocks, int block_k,
@@ -233,8 +233,15 @@ double plan_cost_us(int pair, int bn, int split, long long M, long long N, int k
         const double exchange_us = split == 2 ? 2.5 : (split == 4 ? 6.0 : 13.0);
         clk = main + epi_clk / split + exchange_us * 1900.0;
     } else {
+        // Steady state: a tile's slab stores run beside the next tile's main loop.  When every SM streams C
+        // the stores pace at the HBM write rate, ~1130 clk per 16 KB slab (measured), and the loads of the
+        // main loop share the SM's port with them: fitted, the tile period is the longer of the two plus a
+        // fifth of the shorter (applying it to store-paced tiles only made the model jump at main = store
+        // and pick narrow tiles that re-read A four times as often: 20-30 % slower).
+        const double store_clk = 1130.0 * (bn / 32);
+        const double period = (main > store_clk ? main : store_clk) + 0.2 * (main > store_clk ? store_clk : main);
         const long long waves = (tiles + slots - 1) / slots;
-        clk = static_cast<double>(waves - 1) * (main > epi_clk ? main : epi_clk) + main + epi_clk;
+        clk = static_cast<double>(waves - 1) * period + main + epi_clk;
     }
     return 3.7 + (pair ? 1.0 : 0.0) + clk / 1900.0;   // pairs: cluster launch, two cluster barriers
 }
