@@ -41,7 +41,7 @@ NCU_TRAFFIC_BYTES = {
     "square": 1936e6,   # profiles/dense_kernel_square_sweep.md, latest capture: (2.2 + 8.5 + 53.2 + 607.9 + 9013.4) MB / 5 launches
     "bert": None,
     "resnet": None,
-    "skinny": 58.9e6,   # profiles/skinny_kernel_14336x4096.md: one 14336 x 4096 launch (traffic = algorithmic bytes)
+    "skinny": 33.5e6,   # profiles/skinny_kernel_14336x4096.md: 8839.7 MB over the 264 launches of a step (= algorithmic bytes)
 }
 
 
