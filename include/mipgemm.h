@@ -40,9 +40,9 @@
  * --------------
  * Some calls need global scratch memory (operand re-pitching, slot-padded
  * filters for convolutions gathered in software, the explicit im2col matrix
- * for the few convolutions neither the TMA nor the gather warps can handle).  By default it is taken with cudaMallocAsync on the
- * call's stream and released with cudaFreeAsync after the last kernel of the
- * call.  A caller may instead lend a buffer with mipgemm_set_workspace(); calls
+ * for the few convolutions neither the TMA nor the gather warps can handle).
+ * By default it is taken with cudaMallocAsync on the call's stream and
+ * released with cudaFreeAsync after the last kernel of the call.  A caller may instead lend a buffer with mipgemm_set_workspace(); calls
  * that need more than was lent fail with MIPGEMM_ERR_WORKSPACE.  A lent buffer
  * is shared by all calls: calls that use it must be ordered on one stream.
  */
