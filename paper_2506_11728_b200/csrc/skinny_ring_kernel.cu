@@ -109,9 +109,9 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
     int (*red)[16][17] = reinterpret_cast<int (*)[16][17]>(smem + kRingSlots * kSlotBytes);
     const uint32_t ctrl = ring + kRingSlots * kSlotBytes + kRedBytes;
     const uint32_t bar_full = ctrl, bar_empty = ctrl + 8u * kMaxRingSlots;
+    const uint32_t bar_tokens = ctrl + 16u * kMaxRingSlots + 8u;
     volatile uint32_t* abort_flag =
         reinterpret_cast<volatile uint32_t*>(smem + kRingSlots * kSlotBytes + kRedBytes + 16 * kMaxRingSlots);
-    uint8_t* tok_smem = smem + kRingSlots * kSlotBytes + kRedBytes + kRingCtrlBytes;
     const uint32_t tok_base = ctrl + kRingCtrlBytes;
     const int tok_pitch = p.K + kTokenPad;
 
@@ -122,6 +122,7 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
             mbar_init(bar_full + 8u * s, 1);
             mbar_init(bar_empty + 8u * s, kRingConsumers);
         }
+        mbar_init(bar_tokens, 1);
         *abort_flag = 0;
         fence_mbar_init();
         tma_prefetch_desc(&p.tmap_b);
@@ -172,19 +173,23 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
         const uint32_t sx0 = tok_base + g * tok_pitch, sx1 = tok_base + (g + 8) * tok_pitch;
         const bool tsm = p.tokens_in_smem != 0;
         if (tsm) {
-            // The tokens are read by every unit: one copy per CTA instead of one L2 read per unit.
-            // The consumers make it while the producer's first loads are in flight.
-            const int vecs = p.K >> 4;
-            for (int i = threadIdx.x; i < p.M * vecs; i += kRingConsumers * 32) {
-                const int r = i / vecs, v = i - r * vecs;
-                *reinterpret_cast<uint4*>(tok_smem + r * tok_pitch + v * 16) =
-                    __ldg(reinterpret_cast<const uint4*>(A + static_cast<long long>(r) * p.lda) + v);
+            // The tokens are read by every unit: one copy per CTA instead of one L2 read per unit,
+            // as one bulk copy per token row, all in flight at once (this sits on the critical
+            // path right after the previous kernel's completion, and L2 round trips are long
+            // while every SM streams weights).
+            if (threadIdx.x == 0) {
+                mbar_arrive_expect_tx(bar_tokens, static_cast<uint32_t>(p.M) * static_cast<uint32_t>(p.K));
+                for (int r = 0; r < p.M; ++r)
+                    bulk_load_1d(tok_base + r * tok_pitch, A + static_cast<long long>(r) * p.lda,
+                                 static_cast<uint32_t>(p.K), bar_tokens);
             }
-            asm volatile("bar.sync 1, 256;" ::: "memory");
+            ok = mbar_wait(bar_tokens, 0u, abort_flag, budget);
         }
-        TokenRegs cur, nxt;
-        if (tsm) load_tokens_smem<kSecondTokenBlock>(cur, sx0, sx1, warp, p.K, t, tok0_ok, tok1_ok);
-        else load_tokens<kSecondTokenBlock>(cur, x0, x1, warp, p.K, t, tok0_ok, tok1_ok);
+        TokenRegs cur = {}, nxt;
+        if (ok) {
+            if (tsm) load_tokens_smem<kSecondTokenBlock>(cur, sx0, sx1, warp, p.K, t, tok0_ok, tok1_ok);
+            else load_tokens<kSecondTokenBlock>(cur, x0, x1, warp, p.K, t, tok0_ok, tok1_ok);
+        }
         for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
             int acc0[4] = {0, 0, 0, 0};
             int acc1[4] = {0, 0, 0, 0};
@@ -238,7 +243,13 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
         }
         if (!ok) {
             // Unwinding: every slot the producer may have filled must land before the CTA exits;
-            // wait (bounded) on the barriers that are still pending.
+            // wait (bounded) on the barriers that are still pending, the tokens' first.
+            if (tsm) {
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(bar_tokens, 0u)) {
+                    if (globaltimer_ns() - t0 > 2000000ull) break;
+                }
+            }
             for (int i = 0; i < kRingSlots; ++i) {
                 const uint64_t t0 = globaltimer_ns();
                 const uint32_t si = s + i;
@@ -308,12 +319,13 @@ bool skinny_ring_supported(const SkinnyParams& p, int sm_count) {
     if (!skinny_supported(p)) return false;
     if (p.K % 128 != 0) return false;
     // needs enough 16-row units that (almost) every SM streams; smaller N uses the cluster-split form.
-    // With more than 8 tokens the consumers' token traffic doubles: measured, the ring then only wins
-    // when the tokens fit in shared memory beside the ring and every SM gets several units.
+    // With more than 8 tokens the consumers' token traffic doubles: the ring then only wins when the
+    // tokens fit in shared memory beside it.
     const long long units = (static_cast<long long>(p.N) + 15) / 16;
-    if (p.M <= 8) return units >= sm_count;
+    if (units < sm_count) return false;
+    if (p.M <= 8) return true;
     const long long tok_bytes = static_cast<long long>(p.M) * (p.K + kTokenPad);
-    return units >= 3LL * sm_count && (kRingSmemMax - kRedBytes - kRingCtrlBytes - 1024 - tok_bytes) / kSlotBytes >= 6;
+    return (kRingSmemMax - kRedBytes - kRingCtrlBytes - 1024 - tok_bytes) / kSlotBytes >= 6;
 }
 
 cudaError_t launch_skinny_ring(const SkinnyRingParams& p, int sm_count, cudaStream_t stream) {
