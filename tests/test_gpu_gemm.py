@@ -208,6 +208,21 @@ def test_skinny_with_constant_weights_promise(mg):
         mg.mipgemm_set_weights_constant(0)
 
 
+@pytest.mark.parametrize("promise", [0, 1])
+def test_skinny_ring_slots_reused_with_two_ctas_per_sm(mg, promise):
+    """Few ring slots, several chunks per CTA and two CTAs streaming on every SM: a slot is refilled (an
+    asynchronous write) right after its readers release it, so the release must come after their loads have
+    been performed.  Releasing on the barrier arrive alone gave thousands of wrong columns in these cases."""
+    mg.mipgemm_set_weights_constant(promise)
+    try:
+        for rep in range(3):
+            for i, (M, N, K, acc) in enumerate([(15, 4096, 4096, True), (16, 4096, 4096, False), (4, 5000, 4096, True),
+                                                (16, 14336, 4096, False), (8, 11008, 4096, False), (1, 4096, 11008, False)]):
+                check_case(mg, "s8", M, N, K, seed=900 + 10 * rep + i, accumulate=acc, expect_path=mg.PATH_SKINNY)
+    finally:
+        mg.mipgemm_set_weights_constant(0)
+
+
 def test_skinny_misaligned_falls_back_to_dense(mg):
     path = check_case(mg, "s8", 4, 300, 100, seed=41)
     assert path & mg.PATH_MASK == mg.PATH_DENSE and path & mg.PATH_REPACK
