@@ -1,10 +1,11 @@
 // Skinny-M MIP GEMM, ring form: the weight matrix streams through a deep shared-memory ring
 // filled by the TMA, so that far more bytes are in flight per SM than registers could hold.
 //
-// One persistent CTA per SM.  A work unit is 16 consecutive weight rows (columns j of C) over
+// Persistent CTAs, two per SM with half the shared memory each when at least two ring slots fit
+// beside the tokens, else one.  A work unit is 16 consecutive weight rows (columns j of C) over
 // the whole of K; it arrives as chunks of 16 rows x 1024 bytes, each one TMA load of a
-// rank-3 box {128 B, 16 rows, 8 k-slices} into a 16 KB ring slot (12 slots = 192 KB in flight
-// per SM, every slice 128-byte swizzled so the warps' 16-byte reads are conflict-free).  Warp 8
+// rank-3 box {128 B, 16 rows, 8 k-slices} into a 16 KB ring slot (up to 12 slots = 192 KB in
+// flight per SM, every slice 128-byte swizzled so the warps' 16-byte reads are conflict-free).  Warp 8
 // produces; warps 0-7 consume: warp w multiplies slice w of every chunk by the M tokens with
 // warp-level m16n8k32 integer MMAs (weights are the 16-row operand, tokens the 8-column
 // operand; k positions permuted identically on both sides so that all accesses are 16 bytes),
