@@ -278,10 +278,12 @@ cudaError_t launch_ring_t(SkinnyRingParams p, int grid, cudaStream_t stream) {
     p.tokens_in_smem = (kRingSmemMax - fixed - tok_bytes) / kSlotBytes >= 6 ? 1 : 0;
     int slots = (kRingSmemMax - fixed - (p.tokens_in_smem ? tok_bytes : 0)) / kSlotBytes;
     if (slots > kMaxRingSlots) slots = kMaxRingSlots;
-    // Programmatic dependent launch only under the constant-weights promise (it is what lets the next call's
-    // producer start early).  Without the promise an early CTA has nothing to do but wait, and it measured
-    // 4-9 % slower in long CUDA-graph chains of these kernels.
-    p.pdl_mode = p.b_constant ? 1 : 0;
+    // Programmatic dependent launch: the kernel lets its successor start as soon as all of its own CTAs
+    // are resident.  Under the constant-weights promise the successor's producer then fetches B at once;
+    // without it the successor's CTAs only set up and wait, which still hides their launch and prologue
+    // now that half-memory CTAs leave room for them (2.28 -> 2.21 ms over a chain of 264 decode GEMMs; with
+    // one 210 KB CTA per SM it had measured 4-9 % slower).
+    p.pdl_mode = 1;
     {
         // Two CTAs per SM, each with half the shared memory, whenever at least two ring slots are left
         // beside the tokens: while one CTA reduces and stores a unit (or, under the constant-weights
