@@ -48,7 +48,8 @@ __device__ __forceinline__ void fence_mbar_init() {
 __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async;" ::: "memory");
 }
-// Orders this thread's earlier shared-memory writes before later async-proxy (TMA) reads.
+// Orders this thread's earlier generic-proxy accesses to shared memory (writes a TMA store or an MMA
+// will read; loads from bytes a TMA load will overwrite) before later async-proxy accesses.
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
