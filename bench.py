@@ -607,7 +607,7 @@ def main():
                     "traffic": NCU_TRAFFIC_BYTES.get(args.workload)}
     else:
         achieved = args.steps * step_bytes / (kernel_ms * 1e-3) / 1e9
-        kname = "mip_skinny_kernel" if args.workload == "skinny" else "mip_dense_kernel"
+        kname = "mip_skinny_ring_kernel" if args.workload == "skinny" else "mip_dense_kernel"
         roofline = {"bound": "hbm", "kernel": kname, "achieved": achieved, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                     "peak_source": "%s copy bandwidth" % peaks["_source"],
