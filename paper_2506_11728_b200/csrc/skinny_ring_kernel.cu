@@ -14,7 +14,6 @@
 // never split across CTAs, so there is no scratch, no atomics and no inter-CTA wait; every
 // barrier wait inside the CTA is bounded and reports through the device status word.
 // Requires K % 128 == 0 and 16-byte aligned operands; other shapes use the register form.
-#include <cstdlib>
 #include "internal.h"
 #include "ptx.cuh"
 
