@@ -4,7 +4,7 @@ import pytest
 
 from oracle import mip_oracle as orc
 from paper_2506_11728_b200 import inputs
-from gpu_util import run_gemm, first_mismatch
+from gpu_util import run_gemm, first_mismatch, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -221,6 +221,41 @@ def test_skinny_ring_slots_reused_with_two_ctas_per_sm(mg, promise):
                 check_case(mg, "s8", M, N, K, seed=900 + 10 * rep + i, accumulate=acc, expect_path=mg.PATH_SKINNY)
     finally:
         mg.mipgemm_set_weights_constant(0)
+
+
+@pytest.mark.parametrize("promise", [0, 1])
+@pytest.mark.parametrize("M", [1, 4])
+def test_skinny_chain_of_dependent_launches(mg, M, promise):
+    """Six ring-form launches enqueued back to back, each reading as its tokens the bytes of the previous one's
+    int32 output: a launch that starts under its predecessor's tail (programmatic dependent launch, CTAs of two
+    calls on one SM) must still see that output complete."""
+    import torch
+    N, K0, depth = 4096, 4096, 6
+    K = 4 * N
+    A0 = inputs.uniform_s8(M * K0, 4100 + M)
+    B0 = inputs.uniform_s8(N * K0, 4200 + M)
+    B = inputs.uniform_s8(N * K, 4300 + M)
+    dA0, _k0 = to_dev(A0)
+    dB0, _k1 = to_dev(B0)
+    dB, _k2 = to_dev(B)
+    dC = [torch.full((M * N,), 0x7F7F7F7F, dtype=torch.int32, device="cuda") for _ in range(depth)]
+    torch.cuda.synchronize()
+    mg.mipgemm_set_weights_constant(promise)
+    try:
+        mg.mipgemm_s8s8s32(M, N, K0, dA0, K0, dB0, K0, dC[0], N, False)
+        assert mg.mipgemm_last_path() & mg.PATH_MASK == mg.PATH_SKINNY
+        for d in range(1, depth):
+            mg.mipgemm_s8s8s32(M, N, K, dC[d - 1].view(torch.uint8), K, dB, K, dC[d], N, False)
+    finally:
+        mg.mipgemm_set_weights_constant(0)
+    torch.cuda.synchronize()
+    assert mg.mipgemm_device_status() == mg.OK
+    want = orc.gemm(A0, B0, M, N, K0)
+    for d in range(depth):
+        got = dC[d].cpu().numpy()
+        assert np.array_equal(got, want), "launch %d of the chain: %s" % (d, first_mismatch(got, want))
+        if d + 1 < depth:
+            want = orc.gemm(want.view(np.int8), B, M, N, K)
 
 
 def test_skinny_misaligned_falls_back_to_dense(mg):
