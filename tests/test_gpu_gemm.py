@@ -258,6 +258,35 @@ def test_skinny_chain_of_dependent_launches(mg, M, promise):
             want = orc.gemm(want.view(np.int8), B, M, N, K)
 
 
+@pytest.mark.parametrize("M,N", [(300, 512), (2500, 256), (64, 1024)])
+def test_dense_chain_of_dependent_launches(mg, M, N):
+    """The same for the dense kernel, whose launches also start under their predecessor's tail: the bytes of one
+    launch's int32 output are the next one's A."""
+    import torch
+    K0, depth = 192, 6
+    K = 4 * N
+    A0 = inputs.uniform_s8(M * K0, 4400 + M)
+    B0 = inputs.uniform_s8(N * K0, 4500 + M)
+    B = inputs.uniform_s8(N * K, 4600 + M)
+    dA0, _k0 = to_dev(A0)
+    dB0, _k1 = to_dev(B0)
+    dB, _k2 = to_dev(B)
+    dC = [torch.full((M * N,), 0x7F7F7F7F, dtype=torch.int32, device="cuda") for _ in range(depth)]
+    torch.cuda.synchronize()
+    mg.mipgemm_s8s8s32(M, N, K0, dA0, K0, dB0, K0, dC[0], N, False)
+    for d in range(1, depth):
+        mg.mipgemm_s8s8s32(M, N, K, dC[d - 1].view(torch.uint8), K, dB, K, dC[d], N, False)
+        assert mg.mipgemm_last_path() & mg.PATH_MASK in (mg.PATH_DENSE, mg.PATH_DENSE_PAIR)
+    torch.cuda.synchronize()
+    assert mg.mipgemm_device_status() == mg.OK
+    want = orc.gemm(A0, B0, M, N, K0)
+    for d in range(depth):
+        got = dC[d].cpu().numpy()
+        assert np.array_equal(got, want), "launch %d of the chain: %s" % (d, first_mismatch(got, want))
+        if d + 1 < depth:
+            want = orc.gemm(want.view(np.int8), B, M, N, K)
+
+
 def test_skinny_misaligned_falls_back_to_dense(mg):
     path = check_case(mg, "s8", 4, 300, 100, seed=41)
     assert path & mg.PATH_MASK == mg.PATH_DENSE and path & mg.PATH_REPACK
