@@ -36,6 +36,17 @@
  *  - M == 0 or N == 0: no-op, MIPGEMM_OK.  K == 0: C is zero-filled
  *    (accumulate == 0) or left unchanged (accumulate != 0).
  *
+ * Threads
+ * -------
+ * Entry points may be called from several host threads at once, on the same or on different
+ * streams and devices: per-device set-up is serialised internally, mipgemm_last_path() and
+ * mipgemm_last_cuda_error() are per thread.  Process-wide switches (mipgemm_set_tuning,
+ * mipgemm_set_weights_constant, mipgemm_set_workspace) take effect atomically for calls that
+ * start after they return; they are meant to be set up front, not raced with compute calls.
+ * Calls that share memory must be ordered by the caller as with any CUDA work: a lent workspace
+ * (one stream at a time), the static array of mipgemm_s8s8s32_static_scratch, and the staging
+ * streams of the host-buffer entry points (calls of those are serialised per device).
+ *
  * Scratch memory
  * --------------
  * Some calls need global scratch memory (operand re-pitching, slot-padded
@@ -76,7 +87,7 @@ typedef enum {
     MIPGEMM_PATH_SKINNY = 3,      /* M <= 16 streaming kernel                                */
     MIPGEMM_PATH_TRIVIAL = 4,     /* K == 0 fill or empty problem                            */
     MIPGEMM_PATH_REPACK = 0x100,  /* flag: an operand was re-pitched into scratch first      */
-    MIPGEMM_PATH_SPLITK = 0x200,  /* flag: K was split and reduced with integer atomics      */
+    MIPGEMM_PATH_SPLITK = 0x200,  /* flag: K was split over CTAs (partials added exactly)    */
     MIPGEMM_PATH_IM2COL_TMA = 0x400,   /* flag: conv gathered by TMA im2col loads            */
     MIPGEMM_PATH_IM2COL_EXPLICIT = 0x800, /* flag: conv materialised the augmented matrix    */
     MIPGEMM_PATH_BATCHED = 0x1000,     /* flag: a whole strided batch ran as one launch       */
@@ -222,14 +233,15 @@ int mipgemm_conv_u8s8f32_dequant(int64_t Nb, int64_t H, int64_t W, int64_t Cin, 
 
 /*
  * Host-buffer variants (the end-to-end path): A, B and C are HOST pointers (pinned or
- * pageable) with the same layouts as above.  The call stages the operands into device
- * memory obtained with cudaMallocAsync on `stream`, runs the device entry point, copies
- * the M x N result back into C (padding columns of the host C are left untouched; with
- * accumulate != 0 the host C is uploaded first), releases the device memory and
- * SYNCHRONISES the stream before returning.  Large problems (>= 2048 rows, >= 32 MB) are cut
- * into row blocks that three streams pipeline -- operands in, compute on `stream`, results
- * out -- so both directions of the host link are busy at once; pinned host memory is what
- * makes those copies asynchronous.  Same return codes as the device variants.
+ * pageable) with the same layouts as above.  The call stages the operands into a device
+ * staging buffer, runs the device entry point, copies the M x N result back into C (padding
+ * columns of the host C are left untouched; with accumulate != 0 the host C is uploaded
+ * first) and SYNCHRONISES the stream before returning.  Large problems (>= 32 MB) are cut into
+ * up to 8 x 8 blocks of C that three streams pipeline -- operand blocks in, compute on
+ * `stream`, finished blocks out -- so both directions of the host link are busy at once; pinned
+ * host memory is what makes those copies asynchronous.  The staging buffer (one per device, as
+ * large as the largest call so far) stays allocated between calls; mipgemm_release_staging()
+ * frees it.  Calls on one device run one at a time.  Same return codes as the device variants.
  */
 int mipgemm_host_s8s8s32(int64_t M, int64_t N, int64_t K,
                          const int8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
@@ -268,8 +280,11 @@ int mipgemm_host_u8s8s32(int64_t M, int64_t N, int64_t K,
  *    nothing has to be cleared between calls.  But two calls whose kernels can overlap on
  *    the GPU (different streams, or several host threads) race on the array and corrupt
  *    each other's operands: order such calls on one stream or serialise them yourself.
- *  - A bounded device-side wait that expires in this path sets a word private to this
- *    entry point; mipgemm_device_status() does not report it.
+ *  - A bounded device-side wait that expires in this path sets a status word that is a
+ *    static symbol of the library as well.  mipgemm_static_scratch_status() reads and clears
+ *    it without allocating anything; mipgemm_device_status() reports it too, but that call
+ *    belongs to the regular entry points and allocates their status word on first use.
+ *  - mipgemm_last_path() reports the kernel family as for the regular entry point.
  */
 #define MIPGEMM_STATIC_SCRATCH_BYTES (8u << 20)
 int mipgemm_s8s8s32_static_scratch(int64_t M, int64_t N, int64_t K,
@@ -278,10 +293,28 @@ int mipgemm_s8s8s32_static_scratch(int64_t M, int64_t N, int64_t K,
                                    int32_t *C, int64_t ldc,
                                    int accumulate, void *stream);
 
+/* Companion of the entry point above, equally allocation-free (the paper has no counterpart):
+ * synchronises `stream`, then returns MIPGEMM_OK, or MIPGEMM_ERR_TIMEOUT if a kernel launched by
+ * mipgemm_s8s8s32_static_scratch on the current device gave up a bounded wait since the last query
+ * (C is then incomplete; the flag is cleared), or MIPGEMM_ERR_CUDA. */
+int mipgemm_static_scratch_status(void *stream);
+
+/* Frees the current device's staging buffer of the host-buffer variants (it is allocated again by
+ * the next such call). */
+int mipgemm_release_staging(void);
+
 /* ---- support calls (no counterpart in the paper) ---- */
 
 /* Number of kernels this library has enqueued since it was loaded (all threads, all devices). */
 uint64_t mipgemm_launch_count(void);
+
+/* The library remembers the plan (tile shape, split, pipeline depth) and the encoded TMA tensor maps of
+ * recent dense GEMM / TMA-convolution calls and the weight map of skinny calls, keyed on every argument
+ * that determines them (shapes, pointers, pitches, output transform, device, tuning overrides): a
+ * repeated call skips planning and encoding.  1024 direct-mapped entries, thread-safe; the environment
+ * variable MIPGEMM_PLAN_CACHE=0 switches it off.  Returns 1 if the cache is on, 0 if off, and the
+ * number of calls served from / entered into it since the library was loaded. */
+int mipgemm_plan_cache_stats(uint64_t *hits, uint64_t *misses);
 
 /* Synchronises `stream` and returns MIPGEMM_OK, MIPGEMM_ERR_TIMEOUT if any kernel
  * since the last call gave up a bounded wait (the flag is then cleared), or
@@ -335,9 +368,34 @@ int mipgemm_probe_i8_peak(int iters, int *grid_out, double *ops_per_launch,
  */
 int mipgemm_set_weights_constant(int on);
 
+/*
+ * The same promise for individual buffers (the form an inference runtime uses: register each weight
+ * tensor once after loading it).  A later call with M <= 16 whose B operand lies entirely inside a
+ * registered range [base, base + bytes) is treated as under the promise above, whatever the
+ * process-wide switch says; calls on other buffers are not affected.  Unregister a range (by its
+ * base) before the buffer is freed or rewritten.  Ranges must not overlap.  Thread-safe.
+ * Returns MIPGEMM_OK, or MIPGEMM_ERR_INVALID_ARG (NULL / empty range; unknown base).
+ */
+int mipgemm_register_constant_weights(const void *base, size_t bytes);
+int mipgemm_unregister_constant_weights(const void *base);
+
 /* Overrides for experiments: tile width (0 = heuristic; a multiple of 32 up to 256), pipeline
  * depth (0 = heuristic), split-K factor (0 = heuristic, 1 = off), force path. */
 int mipgemm_set_tuning(int block_n, int stages, int split_k, int force_path);
+
+/*
+ * Test hook for the unwinding path (no counterpart in the paper).  Every device-side wait of the
+ * kernels is bounded (4 s by default); when one runs out, all roles of the CTA leave their loops,
+ * wait -- again bounded -- for copies and MMAs still in flight, release tensor memory and return, and
+ * mipgemm_device_status() reports MIPGEMM_ERR_TIMEOUT.  This call makes that happen on purpose, by
+ * withholding a signal inside the kernel (never by faulting or trapping):
+ *   flags bit 0 : the dense kernel's MMA warp never signals "accumulator ready", so the epilogue warps'
+ *                 wait runs out; the skinny ring kernel's first CTA never loads the second 1 KB k-chunk
+ *                 of its first unit, so its consumer warps' wait runs out.  C is left incomplete.
+ *   wait_budget_ns : limit of every wait in later launches (0 = the default 4 s).
+ * Process-wide; returns MIPGEMM_OK or MIPGEMM_ERR_INVALID_ARG (unknown flag bits).
+ */
+int mipgemm_debug_set(int flags, unsigned long long wait_budget_ns);
 
 #ifdef __cplusplus
 }

@@ -19,7 +19,12 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "mip_oracle.c")
-_LIB = os.path.join(_HERE, "libmip_oracle.so")
+# MIP_ORACLE_SANITIZE=1 selects a second build of the same source with gcc's address and undefined-
+# behaviour sanitizers (-O1), used by the oracle's own unit tests: an out-of-bounds index or a signed
+# overflow inside the oracle then aborts the test process instead of passing by luck.  The process must
+# have the sanitizer runtime preloaded (see sanitizer_env()).
+SANITIZED = os.environ.get("MIP_ORACLE_SANITIZE") == "1"
+_LIB = os.path.join(_HERE, "libmip_oracle_san.so" if SANITIZED else "libmip_oracle.so")
 _lock = threading.Lock()
 _lib = None
 
@@ -30,11 +35,21 @@ def build(force: bool = False) -> str:
         stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
         if force or stale:
             tmp = _LIB + ".tmp.%d" % os.getpid()
-            cmd = ["gcc", "-O3", "-march=native", "-fopenmp", "-fPIC", "-shared",
-                   "-std=c11", "-Wall", "-Wextra", "-o", tmp, _SRC, "-lm"]
+            opt = ["-O1", "-g", "-fsanitize=address,undefined", "-fno-sanitize-recover=undefined",
+                   "-fno-omit-frame-pointer"] if SANITIZED else ["-O3", "-march=native"]
+            cmd = ["gcc"] + opt + ["-fopenmp", "-fPIC", "-shared", "-std=c11", "-Wall", "-Wextra", "-o", tmp, _SRC, "-lm"]
             subprocess.run(cmd, check=True)
             os.replace(tmp, _LIB)
     return _LIB
+
+
+def sanitizer_env() -> dict:
+    """Environment for a child process that should load the sanitized oracle build."""
+    env = dict(os.environ)
+    asan = subprocess.run(["gcc", "-print-file-name=libasan.so"], capture_output=True, text=True, check=True).stdout.strip()
+    env.update(MIP_ORACLE_SANITIZE="1", LD_PRELOAD=asan,
+               ASAN_OPTIONS="detect_leaks=0:abort_on_error=1", UBSAN_OPTIONS="halt_on_error=1:print_stacktrace=1")
+    return env
 
 
 def _load():

@@ -61,6 +61,12 @@ SIGNATURES = {
     "mipgemm_probe_i8_peak": (_int, [_int, ctypes.POINTER(_int), ctypes.POINTER(ctypes.c_double), _vp, _vp]),
     "mipgemm_set_tuning": (_int, [_int, _int, _int, _int]),
     "mipgemm_set_weights_constant": (_int, [_int]),
+    "mipgemm_register_constant_weights": (_int, [_vp, _sz]),
+    "mipgemm_unregister_constant_weights": (_int, [_vp]),
+    "mipgemm_static_scratch_status": (_int, [_vp]),
+    "mipgemm_release_staging": (_int, []),
+    "mipgemm_debug_set": (_int, [_int, ctypes.c_ulonglong]),
+    "mipgemm_plan_cache_stats": (_int, [ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]),
 }
 for _name, (_res, _args) in SIGNATURES.items():
     _fn = getattr(_lib, _name)
@@ -253,6 +259,40 @@ def mipgemm_probe_i8_peak(iters: int, sink, stream=None):
 def mipgemm_set_weights_constant(on) -> int:
     """Promise that B of later M <= 16 calls is never written by work still pending on the stream."""
     return _check(_lib.mipgemm_set_weights_constant(int(bool(on))), True)
+
+
+def mipgemm_register_constant_weights(buf, nbytes: int = 0, check=True) -> int:
+    """Declares [buf, buf + nbytes) constant: M <= 16 calls whose B lies inside it may fetch it early.
+    ``nbytes`` defaults to the tensor's size."""
+    if not nbytes and hasattr(buf, "numel"):
+        nbytes = buf.numel() * buf.element_size()
+    return _check(_lib.mipgemm_register_constant_weights(_ptr(buf), nbytes), check)
+
+
+def mipgemm_unregister_constant_weights(buf, check=True) -> int:
+    return _check(_lib.mipgemm_unregister_constant_weights(_ptr(buf)), check)
+
+
+def mipgemm_release_staging() -> int:
+    """Frees the device staging buffer the host-buffer entry points keep between calls."""
+    return _check(_lib.mipgemm_release_staging(), True)
+
+
+def mipgemm_debug_set(flags=0, wait_budget_ns=0) -> int:
+    """Test hook: withhold a device-side signal (bit 0) and set the limit of device-side waits (0 = 4 s)."""
+    return _check(_lib.mipgemm_debug_set(int(flags), int(wait_budget_ns)), True)
+
+
+def mipgemm_plan_cache_stats():
+    """(enabled, hits, misses) of the plan / tensor-map cache."""
+    hits, misses = ctypes.c_uint64(0), ctypes.c_uint64(0)
+    on = _lib.mipgemm_plan_cache_stats(ctypes.byref(hits), ctypes.byref(misses))
+    return bool(on), hits.value, misses.value
+
+
+def mipgemm_static_scratch_status(stream=None) -> int:
+    """Allocation-free status query of mipgemm_s8s8s32_static_scratch (synchronises the stream)."""
+    return _lib.mipgemm_static_scratch_status(_stream(stream))
 
 
 def mipgemm_set_tuning(block_n=0, stages=0, split_k=0, force_path=0) -> int:

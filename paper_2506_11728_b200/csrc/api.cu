@@ -6,6 +6,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <atomic>
+#include <map>
 #include <mutex>
 
 #include "../../include/mipgemm.h"
@@ -23,15 +24,48 @@ thread_local float tl_out_scale = 1.0f;
 // ... or requantisation to 8-bit codes (the *_requant entry points): clamp bounds; C then holds bytes
 thread_local int tl_out_q8 = 0, tl_q_lo = 0, tl_q_hi = 0;
 
+// Experiment overrides (mipgemm_set_tuning).  The four values travel in one atomic word, so a call
+// that runs while another thread changes them sees either the old set or the new one, never a mix.
 struct Tuning {
     int block_n = 0, stages = 0, split_k = 0, force_path = 0;
 };
-Tuning g_tuning;
+std::atomic<uint64_t> g_tuning_word{0};
+std::atomic<uint32_t> g_tuning_epoch{0};   // bumped by every change (cached plans remember it)
+uint64_t pack_tuning(const Tuning& t) {
+    return static_cast<uint64_t>(t.block_n & 0xFFFF) | (static_cast<uint64_t>(t.stages & 0xFF) << 16) |
+           (static_cast<uint64_t>(t.split_k & 0xFFFF) << 24) | (static_cast<uint64_t>(t.force_path & 0xFFFFFF) << 40);
+}
+Tuning tuning_now() {
+    const uint64_t w = g_tuning_word.load(std::memory_order_acquire);
+    Tuning t;
+    t.block_n = static_cast<int>(w & 0xFFFF);
+    t.stages = static_cast<int>((w >> 16) & 0xFF);
+    t.split_k = static_cast<int>((w >> 24) & 0xFFFF);
+    t.force_path = static_cast<int>((w >> 40) & 0xFFFFFF);
+    return t;
+}
 bool g_tuning_no_cluster_split = false;  // MIPGEMM_NO_CLUSTER_SPLIT=1: split-K through zero fill + TMA reduce-add
 bool g_tuning_no_skinny_ring = false;    // MIPGEMM_NO_SKINNY_RING=1: always the register form of the skinny kernel
 bool g_tuning_no_tma_store = false;   // MIPGEMM_DIRECT_STORE=1: force the direct-store epilogue
 std::atomic<uint64_t> g_launches{0};
+// Limit of every device-side wait and the test-hook bits handed to the kernels (mipgemm_debug_set).
+std::atomic<unsigned long long> g_wait_budget_ns{4000000000ull};
+std::atomic<int> g_debug_flags{0};
 std::atomic<int> g_weights_constant{0};  // mipgemm_set_weights_constant
+
+// Address ranges the caller has declared constant (mipgemm_register_constant_weights): start -> end.
+std::map<uintptr_t, uintptr_t> g_constant_ranges;
+std::atomic<int> g_constant_range_count{0};
+std::mutex g_ranges_mutex;
+bool inside_constant_range(const void* ptr, size_t bytes) {
+    if (g_constant_range_count.load(std::memory_order_acquire) == 0) return false;
+    const uintptr_t lo = reinterpret_cast<uintptr_t>(ptr), hi = lo + bytes;
+    std::lock_guard<std::mutex> lock(g_ranges_mutex);
+    auto it = g_constant_ranges.upper_bound(lo);     // first range that starts after lo
+    if (it == g_constant_ranges.begin()) return false;
+    --it;
+    return it->first <= lo && hi <= it->second;
+}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -43,6 +77,8 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr int kMaxDevices = 64;
+constexpr int kHostBlocks = 8;                                    // host-buffer calls: up to 8 x 8 blocks of C
+constexpr int kHostEvents = 2 * kHostBlocks + kHostBlocks * kHostBlocks + 3;
 struct DeviceState {
     bool ready = false;
     int status = MIPGEMM_OK;
@@ -50,6 +86,11 @@ struct DeviceState {
     int pair_clusters = 0;                 // co-resident 2-CTA clusters of the pair kernel
     unsigned int* status_word = nullptr;   // device
     cudaStream_t copy_in = nullptr, copy_out = nullptr;   // helper streams of the host-buffer entry points
+    std::mutex host_mutex;                 // host-buffer calls on one device run one at a time
+    void* staging = nullptr;               // their device staging buffer (grow-only) ...
+    size_t staging_bytes = 0;
+    cudaEvent_t host_events[kHostEvents] = {};   // ... and their event pool
+    bool host_events_ready = false;
     void* lent = nullptr;
     size_t lent_bytes = 0;
 };
@@ -58,16 +99,63 @@ std::mutex g_mutex;
 EncodeTiledFn g_encode_tiled = nullptr;
 EncodeIm2colFn g_encode_im2col = nullptr;
 
+struct NoAllocDevice {
+    bool ready = false;
+    int status = MIPGEMM_OK;
+    DeviceState st;                 // sm_count, pair_clusters, status_word (-> g_static_status)
+    unsigned char* scratch = nullptr;   // device address of g_static_scratch on this device
+};
+NoAllocDevice g_noalloc[kMaxDevices];
+std::mutex g_noalloc_mutex;
+
+// MIPGEMM_LOG=1: one line per call on stderr with the dispatch decision.
+bool log_enabled() {
+    static const bool on = env_int("MIPGEMM_LOG", 0) != 0;
+    return on;
+}
+struct Plan;
+void log_dense(const char* what, long long M, long long N, long long K, const Plan& pl, const DenseParams& p, bool hit);
+
 int cuda_fail(cudaError_t e) {
     tl_last_cuda_error = static_cast<int>(e);
     return MIPGEMM_ERR_CUDA;
 }
+
+// Reads a device status word and clears it when set (the caller has synchronised the work that may
+// have written it).  Returns MIPGEMM_OK, MIPGEMM_ERR_TIMEOUT or MIPGEMM_ERR_CUDA.
+int take_status_word(unsigned int* dev_word) {
+    unsigned int word = 0;
+    cudaError_t e = cudaMemcpy(&word, dev_word, sizeof(word), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (word != 0) {
+        e = cudaMemset(dev_word, 0, sizeof(word));
+        if (e != cudaSuccess) return cuda_fail(e);
+        return MIPGEMM_ERR_TIMEOUT;
+    }
+    return MIPGEMM_OK;
+}
+
+// ---- state of the allocation-free entry point (mipgemm_s8s8s32_static_scratch, end of this file)
+// The scratch itself.  Host code must never use this name as an address: on the host it is
+// only a handle for cudaGetSymbolAddress (see noalloc_device()).
+static __device__ __align__(256) unsigned char g_static_scratch[MIPGEMM_STATIC_SCRATCH_BYTES];
+// Word that receives the "bounded wait expired" flag of kernels launched from that path; read and
+// cleared by mipgemm_static_scratch_status() and by mipgemm_device_status().
+static __device__ unsigned int g_static_status;
 
 // Once per device: capability check, driver entry points, kernel attributes, status word.
 int get_device(DeviceState** out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(e);
+    // The tensor-map encoders are driver calls and need the device's context current on the calling
+    // thread; a host thread that has made no runtime call yet has none (cudaGetDevice does not bind it,
+    // cudaSetDevice does).
+    thread_local int tl_context_bound = -1;
+    if (tl_context_bound != dev) {
+        if ((e = cudaSetDevice(dev)) != cudaSuccess) return cuda_fail(e);
+        tl_context_bound = dev;
+    }
     if (dev < 0 || dev >= kMaxDevices) return MIPGEMM_ERR_UNSUPPORTED;
     std::lock_guard<std::mutex> lock(g_mutex);
     DeviceState& d = g_dev[dev];
@@ -249,6 +337,7 @@ double plan_cost_us(int pair, int bn, int split, long long M, long long N, int k
 Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceState* dev, int min_bn = 64,
                int min_bn_pair = 64, bool one_cta_no_split = false) {
     const int sm_count = dev->sm_count;
+    const Tuning tun = tuning_now();
     Plan pl{};
     pl.k_blocks = static_cast<int>((K + block_k - 1) / block_k);
 
@@ -258,13 +347,13 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
     int best_pair = 0, best_bn = 128, best_split = 1;
     double best = 1e30;
     // (an explicit split reduces int32 tiles in global memory, which a float output cannot share)
-    const bool explicit_split = g_tuning.split_k != 0 && !tl_out_f32 && !tl_out_q8;
+    const bool explicit_split = tun.split_k != 0 && !tl_out_f32 && !tl_out_q8;
     // (N-contiguous B tiles come in 128-column blocks per CTA: a forced width must respect that)
-    const int forced_bn = (g_tuning.block_n && (min_bn <= 64 || g_tuning.block_n == 256)) ? g_tuning.block_n : 0;
+    const int forced_bn = (tun.block_n && (min_bn <= 64 || tun.block_n == 256)) ? tun.block_n : 0;
     for (int pair = 0; pair <= 1; ++pair) {
         if (pair && (dev->pair_clusters <= 0 || one_cta_no_split)) continue;
-        if (g_tuning.force_path == MIPGEMM_PATH_DENSE_PAIR && !pair && dev->pair_clusters > 0) continue;
-        if (g_tuning.force_path == MIPGEMM_PATH_DENSE && pair) continue;
+        if (tun.force_path == MIPGEMM_PATH_DENSE_PAIR && !pair && dev->pair_clusters > 0) continue;
+        if (tun.force_path == MIPGEMM_PATH_DENSE && pair) continue;
         for (int bn = 64; bn <= 256; bn += 32) {      // any multiple of 32 columns is a legal tile width
             int bn_use = bn;
             if (bn < (pair ? min_bn_pair : min_bn)) continue;
@@ -304,11 +393,11 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
     const int stage_bytes = kBlockM * block_k + (pl.pair ? bn / 2 : bn) * block_k;
     int stages = (kSmemBudget - kCtrlBytes - kStagingBytes - 1024) / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
-    if (g_tuning.stages) stages = g_tuning.stages < stages ? g_tuning.stages : stages;
+    if (tun.stages) stages = tun.stages < stages ? tun.stages : stages;
     if (stages < 2) stages = 2;
     pl.stages = stages;
 
-    int split = (explicit_split && !one_cta_no_split) ? g_tuning.split_k : best_split;
+    int split = (explicit_split && !one_cta_no_split) ? tun.split_k : best_split;
     if (pl.pair) split = 1;
     if (split > pl.k_blocks) split = pl.k_blocks;
     if (split < 1) split = 1;
@@ -329,6 +418,14 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
     return pl;
 }
 
+void log_dense(const char* what, long long M, long long N, long long K, const Plan& pl, const DenseParams& p, bool hit) {
+    std::fprintf(stderr,
+                 "mipgemm: %s M=%lld N=%lld K=%lld -> dense %s tile=%dx%d k_block=%d stages=%d split_k=%d%s c_mode=%d%s%s plan=%s\n",
+                 what, M, N, K, pl.pair ? "cta-pair" : "one-cta", pl.pair ? 2 * kBlockM : kBlockM, pl.block_n, p.block_k,
+                 pl.stages, pl.split_k, pl.cluster_split ? " (cluster)" : "", p.c_mode, p.accumulate ? " accumulate" : "",
+                 p.out_f32 ? " f32-out" : (p.out_q8 ? " q8-out" : ""), hit ? "cached" : "new");
+}
+
 void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32_t* C, long long ldc,
                  int block_k, bool a_unsigned, int accumulate, DeviceState* dev) {
     p.C = C;
@@ -344,7 +441,12 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
     p.split_k = pl.split_k;
     p.kb_per_split = pl.kb_per_split;
     p.cluster_split = pl.cluster_split;
-    p.group_n = 8;
+    const int group_env = MIP_ENV_KNOB("MIPGEMM_GROUP_N", 0);
+    const int raster_env = MIP_ENV_KNOB("MIPGEMM_RASTER", 0);
+    const int evict_env = MIP_ENV_KNOB("MIPGEMM_C_EVICT_FIRST", 0);
+    p.group_n = group_env > 0 ? group_env : 8;
+    p.raster = raster_env;
+    p.c_evict_first = evict_env;
     p.use_red = (pl.split_k > 1 && !pl.cluster_split) ? 1 : 0;
     p.accumulate = p.use_red ? 0 : (accumulate ? 1 : 0);
     const uintptr_t c_addr = reinterpret_cast<uintptr_t>(C);
@@ -386,7 +488,8 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
     }
     p.a_im2col = 0;
     p.status = dev->status_word;
-    p.wait_budget_ns = 4000000000ull;
+    p.wait_budget_ns = g_wait_budget_ns.load(std::memory_order_relaxed);
+    p.debug_flags = g_debug_flags.load(std::memory_order_relaxed);
     p.trace = nullptr;
 #ifdef MIPGEMM_TRACE
     if (const char* tr = std::getenv("MIPGEMM_TRACE_PTR"))
@@ -394,8 +497,65 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
 #endif
 }
 
+// Plan + encoded tensor maps of recent calls, keyed on everything that determines them (shapes,
+// pointers, pitches, output transform, device, tuning epoch): a repeated call -- the normal case in
+// inference, where the same layer runs on the same buffers again and again -- skips the planner and
+// the three tensor-map encodings and goes straight to the launch.  Direct-mapped, behind a mutex;
+// MIPGEMM_PLAN_CACHE=0 switches it off.
+struct PlanKey {
+    uint64_t w[28];
+};
+struct PlanEntry {
+    bool used = false;
+    PlanKey key;
+    DenseParams p;
+    Plan pl;
+};
+constexpr int kPlanCacheSlots = 1024;
+PlanEntry* g_plan_cache = nullptr;
+std::mutex g_plan_mutex;
+std::atomic<uint64_t> g_plan_hits{0}, g_plan_misses{0};
+bool plan_cache_enabled() {
+    static const int on = env_int("MIPGEMM_PLAN_CACHE", 1);
+#ifdef MIPGEMM_TRACE
+    return false;
+#else
+    return on != 0 && !live_env();
+#endif
+}
+size_t plan_slot(const PlanKey& k) {
+    uint64_t h = 1469598103934665603ull;
+    for (uint64_t v : k.w) { h ^= v; h *= 1099511628211ull; h ^= h >> 29; }
+    return static_cast<size_t>(h % kPlanCacheSlots);
+}
+bool plan_lookup(const PlanKey& k, DenseParams* p, Plan* pl) {
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    if (!g_plan_cache) return false;
+    const PlanEntry& e = g_plan_cache[plan_slot(k)];
+    if (!e.used || std::memcmp(&e.key, &k, sizeof(k)) != 0) return false;
+    *p = e.p;
+    *pl = e.pl;
+    return true;
+}
+void plan_store(const PlanKey& k, const DenseParams& p, const Plan& pl) {
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    if (!g_plan_cache) g_plan_cache = new PlanEntry[kPlanCacheSlots];
+    PlanEntry& e = g_plan_cache[plan_slot(k)];
+    e.used = true;
+    e.key = k;
+    e.p = p;
+    e.pl = pl;
+}
+uint64_t out_mode_word() {
+    uint32_t scale_bits;
+    std::memcpy(&scale_bits, &tl_out_scale, 4);
+    return static_cast<uint64_t>(scale_bits) | (static_cast<uint64_t>(tl_out_f32 & 1) << 32) |
+           (static_cast<uint64_t>(tl_out_q8 & 1) << 33) | (static_cast<uint64_t>(tl_q_lo & 0x1FF) << 34) |
+           (static_cast<uint64_t>(tl_q_hi & 0x1FF) << 43);
+}
+
 int run_dense(DenseParams& p, const Plan& pl, long long M, long long N, int32_t* C, long long ldc,
-              int accumulate, DeviceState* dev, cudaStream_t stream) {
+              int accumulate, DeviceState* dev, cudaStream_t stream, bool c_map_ready = false) {
     if (pl.split_k > 1 && !pl.cluster_split && !accumulate) {
         cudaError_t e = launch_fill_zero(C, ldc, M, N, stream);
         ++g_launches;
@@ -405,7 +565,7 @@ int run_dense(DenseParams& p, const Plan& pl, long long M, long long N, int32_t*
     const int b_rows = pl.pair ? pl.block_n / 2 : pl.block_n;
     const size_t smem = static_cast<size_t>(pl.stages) * (kBlockM * p.block_k + b_rows * p.block_k) +
                         kStagingBytes + kCtrlBytes + 1024;
-    if (p.c_mode == 1 || p.c_mode == 2) {
+    if ((p.c_mode == 1 || p.c_mode == 2) && !c_map_ready) {
         cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(M)};
         cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldc) * 4};
         cuuint32_t box[2] = {32, static_cast<cuuint32_t>(p.c_mode == 1 ? 128 : 32)};
@@ -449,6 +609,7 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
               int64_t ldb, int32_t* C, int64_t ldc, int accumulate, void* stream_v, int path_flags,
               Scratch* outer = nullptr) {
     tl_last_path = MIPGEMM_PATH_NONE;
+    const Tuning tun = tuning_now();
     if (M < 0 || N < 0 || K < 0) return MIPGEMM_ERR_INVALID_ARG;
     if (M > 0x7FFFFF00LL || N > 0x7FFFFF00LL) return MIPGEMM_ERR_INVALID_ARG;
     if (lda < K || ldb < K || ldc < N) return MIPGEMM_ERR_INVALID_ARG;
@@ -482,33 +643,64 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     }
 
     // ---- skinny path
-    if (M <= 16 && !tl_out_q8 && g_tuning.force_path != MIPGEMM_PATH_DENSE &&
-        g_tuning.force_path != MIPGEMM_PATH_DENSE_PAIR) {
+    if (M <= 16 && !tl_out_q8 && tun.force_path != MIPGEMM_PATH_DENSE &&
+        tun.force_path != MIPGEMM_PATH_DENSE_PAIR) {
         SkinnyParams sp{A, lda, B, ldb, C, ldc, static_cast<int>(M), static_cast<int>(N),
                         static_cast<int>(K), a_unsigned ? 1 : 0, accumulate ? 1 : 0, tl_out_f32, tl_out_scale};
         if (skinny_ring_supported(sp, dev->sm_count) && !g_tuning_no_skinny_ring) {
             SkinnyRingParams rp;
             std::memset(&rp, 0, sizeof(rp));
-            cuuint64_t dims[3] = {128, static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(K / 128)};
-            cuuint64_t strides[2] = {static_cast<cuuint64_t>(ldb), 128};
-            cuuint32_t box[3] = {128, 16, 8};
-            cuuint32_t estr[3] = {1, 1, 1};
-            CUresult r = g_encode_tiled(&rp.tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(B), dims,
-                                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            // the weight matrix's tensor map is remembered like a dense plan (kind 3: only tmap_b is used)
+            PlanKey key;
+            DenseParams cached;
+            Plan unused;
+            bool hit = false;
+            if (plan_cache_enabled()) {
+                std::memset(&key, 0, sizeof(key));
+                const uint64_t words[] = {3, reinterpret_cast<uint64_t>(dev), reinterpret_cast<uint64_t>(B),
+                                          static_cast<uint64_t>(ldb), static_cast<uint64_t>(N), static_cast<uint64_t>(K)};
+                std::memcpy(key.w, words, sizeof(words));
+                hit = plan_lookup(key, &cached, &unused);
+            }
+            CUresult r = CUDA_SUCCESS;
+            if (hit) {
+                ++g_plan_hits;
+                rp.tmap_b = cached.tmap_b;
+            } else {
+                cuuint64_t dims[3] = {128, static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(K / 128)};
+                cuuint64_t strides[2] = {static_cast<cuuint64_t>(ldb), 128};
+                cuuint32_t box[3] = {128, 16, 8};
+                cuuint32_t estr[3] = {1, 1, 1};
+                r = g_encode_tiled(&rp.tmap_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(B), dims,
+                                   strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                if (r == CUDA_SUCCESS && plan_cache_enabled()) {
+                    ++g_plan_misses;
+                    std::memset(&cached, 0, sizeof(cached));
+                    cached.tmap_b = rp.tmap_b;
+                    plan_store(key, cached, Plan{});
+                }
+            }
             if (r == CUDA_SUCCESS) {   // (a driver that refuses the overlapping strides: register form below)
                 rp.A = A; rp.lda = lda; rp.C = C; rp.ldc = ldc;
                 rp.M = static_cast<int>(M); rp.N = static_cast<int>(N); rp.K = static_cast<int>(K);
                 rp.a_unsigned = a_unsigned ? 1 : 0; rp.accumulate = accumulate ? 1 : 0;
                 rp.out_f32 = tl_out_f32; rp.out_scale = tl_out_scale;
-                rp.b_constant = g_weights_constant.load();
+                rp.b_constant = (g_weights_constant.load() ||
+                                 inside_constant_range(B, static_cast<size_t>(N - 1) * ldb + K)) ? 1 : 0;
                 rp.status = dev->status_word;
-                rp.wait_budget_ns = 4000000000ull;
+                rp.wait_budget_ns = g_wait_budget_ns.load(std::memory_order_relaxed);
+                rp.debug_flags = g_debug_flags.load(std::memory_order_relaxed);
                 cudaError_t e = launch_skinny_ring(rp, dev->sm_count, stream);
                 ++g_launches;
                 if (e != cudaSuccess) return cuda_fail(e);
                 tl_last_path = MIPGEMM_PATH_SKINNY | path_flags;
+                if (log_enabled())
+                    std::fprintf(stderr, "mipgemm: gemm %s M=%lld N=%lld K=%lld -> skinny ring%s map=%s\n",
+                                 a_unsigned ? "u8" : "s8", static_cast<long long>(M), static_cast<long long>(N),
+                                 static_cast<long long>(K), rp.b_constant ? " (constant weights: early fetch)" : "",
+                                 hit ? "cached" : "new");
                 return MIPGEMM_OK;
             }
             tl_last_cuda_error = 100000 + static_cast<int>(r);
@@ -518,6 +710,10 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
             ++g_launches;
             if (e != cudaSuccess) return cuda_fail(e);
             tl_last_path = MIPGEMM_PATH_SKINNY | path_flags;
+            if (log_enabled())
+                std::fprintf(stderr, "mipgemm: gemm %s M=%lld N=%lld K=%lld -> skinny register form\n",
+                             a_unsigned ? "u8" : "s8", static_cast<long long>(M), static_cast<long long>(N),
+                             static_cast<long long>(K));
             return MIPGEMM_OK;
         }
     }
@@ -552,17 +748,44 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     }
 
     const int block_k = 128;
-    const Plan pl = make_plan(M, N, K, block_k, dev);
+    Plan pl;
     DenseParams p;
-    std::memset(&p, 0, sizeof(p));
-    fill_common(p, pl, M, N, C, ldc, block_k, a_unsigned, accumulate, dev);
-    if ((st = encode_tiled_2d(&p.tmap_a, a_use, K, M, lda_use, block_k, kBlockM)) != MIPGEMM_OK) return st;
-    if ((st = encode_tiled_2d(&p.tmap_b, b_use, K, N, ldb_use, block_k, pl.pair ? pl.block_n / 2 : pl.block_n)) !=
-        MIPGEMM_OK)
-        return st;
-    if ((st = run_dense(p, pl, M, N, C, ldc, accumulate, dev, stream)) != MIPGEMM_OK) return st;
+    // operands used in place: the plan and the tensor maps depend on nothing but the arguments
+    const bool cacheable = plan_cache_enabled() && !repack_a && !repack_b;
+    PlanKey key;
+    bool hit = false;
+    if (cacheable) {
+        std::memset(&key, 0, sizeof(key));
+        const uint64_t words[] = {1, reinterpret_cast<uint64_t>(dev), g_tuning_epoch.load(std::memory_order_acquire),
+                                  static_cast<uint64_t>(a_unsigned) | (accumulate ? 2u : 0u), out_mode_word(),
+                                  static_cast<uint64_t>(M), static_cast<uint64_t>(N), static_cast<uint64_t>(K),
+                                  reinterpret_cast<uint64_t>(A), static_cast<uint64_t>(lda),
+                                  reinterpret_cast<uint64_t>(B), static_cast<uint64_t>(ldb),
+                                  reinterpret_cast<uint64_t>(C), static_cast<uint64_t>(ldc)};
+        std::memcpy(key.w, words, sizeof(words));
+        hit = plan_lookup(key, &p, &pl);
+    }
+    if (hit) {
+        ++g_plan_hits;
+    } else {
+        pl = make_plan(M, N, K, block_k, dev);
+        std::memset(&p, 0, sizeof(p));
+        fill_common(p, pl, M, N, C, ldc, block_k, a_unsigned, accumulate, dev);
+        if ((st = encode_tiled_2d(&p.tmap_a, a_use, K, M, lda_use, block_k, kBlockM)) != MIPGEMM_OK) return st;
+        if ((st = encode_tiled_2d(&p.tmap_b, b_use, K, N, ldb_use, block_k, pl.pair ? pl.block_n / 2 : pl.block_n)) !=
+            MIPGEMM_OK)
+            return st;
+    }
+    if ((st = run_dense(p, pl, M, N, C, ldc, accumulate, dev, stream, hit)) != MIPGEMM_OK) return st;
+    if (cacheable && !hit) {
+        ++g_plan_misses;
+        plan_store(key, p, pl);
+    }
     if (pl.split_k > 1) path_flags |= MIPGEMM_PATH_SPLITK;
     tl_last_path = (pl.pair ? MIPGEMM_PATH_DENSE_PAIR : MIPGEMM_PATH_DENSE) | path_flags;
+    if (log_enabled())
+        log_dense(repack_a || repack_b ? (a_unsigned ? "gemm u8 (re-pitched)" : "gemm s8 (re-pitched)")
+                                       : (a_unsigned ? "gemm u8" : "gemm s8"), M, N, K, pl, p, hit);
     return MIPGEMM_OK;
 }
 
@@ -743,12 +966,13 @@ int batched_impl(bool a_unsigned, int64_t batch, int64_t M, int64_t N, int64_t K
     }
 
     const int block_k = K <= 64 ? 64 : 128;
+    const Tuning tun = tuning_now();
     Plan pl{};
     pl.k_blocks = static_cast<int>((K + block_k - 1) / block_k);
     double best = 1e30;
     for (int bn = 64; bn <= 256; bn *= 2) {
-        if (g_tuning.block_n && bn != 64) continue;
-        const int bn_use = g_tuning.block_n ? g_tuning.block_n : bn;
+        if (tun.block_n && bn != 64) continue;
+        const int bn_use = tun.block_n ? tun.block_n : bn;
         const double us = plan_cost_us(0, bn_use, 1, tiles_m * batch * kBlockM, N, pl.k_blocks, block_k, dev);
         if (us < best) { best = us; pl.block_n = bn_use; }
     }
@@ -805,7 +1029,17 @@ int batched_impl(bool a_unsigned, int64_t batch, int64_t M, int64_t N, int64_t K
     return MIPGEMM_OK;
 }
 
-// Host-buffer front end: stage operands, run the device entry point, copy C back.
+// Pitched copy that degenerates to one flat copy when both sides are dense (flat copies run at the
+// full rate of the host link; pitched ones are slower even when their pitches equal the width).
+cudaError_t copy_rows(void* dst, size_t dpitch, const void* src, size_t spitch, size_t width, size_t rows,
+                      cudaMemcpyKind kind, cudaStream_t stream) {
+    if (rows == 0 || width == 0) return cudaSuccess;
+    if (dpitch == width && spitch == width) return cudaMemcpyAsync(dst, src, width * rows, kind, stream);
+    return cudaMemcpy2DAsync(dst, dpitch, src, spitch, width, rows, kind, stream);
+}
+
+// Host-buffer front end: stage operands, run the device entry point, copy C back.  Calls are serialised
+// per device (they share the staging buffer, the two copy streams and the event pool).
 int host_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, int64_t lda, const int8_t* B,
               int64_t ldb, int32_t* C, int64_t ldc, int accumulate, void* stream_v) {
     if (M < 0 || N < 0 || K < 0 || lda < K || ldb < K || ldc < N) return MIPGEMM_ERR_INVALID_ARG;
@@ -821,110 +1055,128 @@ int host_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     const size_t a_bytes = align256(static_cast<size_t>(M) * pitch);
     const size_t b_bytes = align256(static_cast<size_t>(N) * pitch);
     const size_t c_bytes = align256(static_cast<size_t>(M) * ldc_dev * 4);
-    char* base = nullptr;
-    cudaError_t e = cudaMallocAsync(reinterpret_cast<void**>(&base), a_bytes + b_bytes + c_bytes, stream);
-    if (e != cudaSuccess) {
-        tl_last_cuda_error = static_cast<int>(e);
-        (void)cudaGetLastError();
-        return MIPGEMM_ERR_WORKSPACE;
+    std::lock_guard<std::mutex> host_lock(dev->host_mutex);
+    cudaError_t e;
+    // The staging buffer lives across calls and only grows (mipgemm_release_staging() frees it): taking
+    // gigabytes from the allocator per call cost milliseconds.  Every earlier user has synchronised.
+    if (dev->staging_bytes < a_bytes + b_bytes + c_bytes) {
+        if (dev->staging) (void)cudaFree(dev->staging);
+        dev->staging = nullptr;
+        dev->staging_bytes = 0;
+        e = cudaMalloc(&dev->staging, a_bytes + b_bytes + c_bytes);
+        if (e != cudaSuccess) {
+            tl_last_cuda_error = static_cast<int>(e);
+            (void)cudaGetLastError();
+            return MIPGEMM_ERR_WORKSPACE;
+        }
+        dev->staging_bytes = a_bytes + b_bytes + c_bytes;
     }
+    char* base = static_cast<char*>(dev->staging);
     char* dA = base;
     char* dB = base + a_bytes;
     int32_t* dC = reinterpret_cast<int32_t*>(base + a_bytes + b_bytes);
     st = MIPGEMM_OK;
+    auto check = [&](cudaError_t ee) -> bool {
+        if (ee != cudaSuccess && st == MIPGEMM_OK) st = cuda_fail(ee);
+        return ee == cudaSuccess;
+    };
 
-    // Large problems are cut into row blocks of A and C, and three streams work on them at once: one
-    // copies operands in, the caller's stream computes, one copies results out, so that the two copy
-    // directions of the link overlap each other and the kernels.
+    // Large problems are cut into a grid of up to 8 x 8 blocks of C (1024 rows / columns or more each), and three streams work on them at
+    // once: one copies row blocks of A and column blocks of B in (in the order the blocks of C need them),
+    // the caller's stream computes block after block, one copies finished blocks out -- so both directions
+    // of the host link are busy while the kernels run, and the first block starts after two operand
+    // blocks have arrived instead of after all of B.
     const long long total_bytes = static_cast<long long>(M) * K + static_cast<long long>(N) * K +
                                   4LL * M * N * (accumulate ? 2 : 1);
-    int chunks = 1;
-    if (K > 0 && M >= 2048 && total_bytes >= (32LL << 20) && dev->copy_in && dev->copy_out) {
-        chunks = static_cast<int>(M / 1024);
-        if (chunks > 8) chunks = 8;
+    int bi = 1, bj = 1;
+    if (K > 0 && total_bytes >= (32LL << 20) && dev->copy_in && dev->copy_out) {
+        bi = static_cast<int>(M / 1024 < 1 ? 1 : (M / 1024 > kHostBlocks ? kHostBlocks : M / 1024));
+        bj = static_cast<int>(N / 1024 < 1 ? 1 : (N / 1024 > kHostBlocks ? kHostBlocks : N / 1024));
+        static const int max_bi = env_int("MIPGEMM_HOST_ROW_BLOCKS", kHostBlocks);
+        static const int max_bj = env_int("MIPGEMM_HOST_COL_BLOCKS", kHostBlocks);
+        if (bi > max_bi) bi = max_bi < 1 ? 1 : max_bi;
+        if (bj > max_bj) bj = max_bj < 1 ? 1 : max_bj;
     }
-    if (chunks > 1) {
-        const long long rows_per = round_up((M + chunks - 1) / chunks, 256);
-        chunks = static_cast<int>((M + rows_per - 1) / rows_per);
-        cudaEvent_t ev[4 + 2 * 8];     // start, B, done-in, done-out and two per row block
+    if (bi * bj > 1) {
+        if (!dev->host_events_ready) {
+            for (int i = 0; i < kHostEvents; ++i)
+                if (!check(cudaEventCreateWithFlags(&dev->host_events[i], cudaEventDisableTiming))) return st;
+            dev->host_events_ready = true;
+        }
         int n_ev = 0;
-        auto new_event = [&](cudaEvent_t* out) -> bool {
-            cudaError_t ee = cudaEventCreateWithFlags(out, cudaEventDisableTiming);
-            if (ee != cudaSuccess) { st = cuda_fail(ee); return false; }
-            ev[n_ev++] = *out;
-            return true;
-        };
-        auto check = [&](cudaError_t ee) -> bool {
-            if (ee != cudaSuccess && st == MIPGEMM_OK) st = cuda_fail(ee);
-            return ee == cudaSuccess;
-        };
-        cudaEvent_t ev_start = nullptr, ev_b = nullptr, ev_done = nullptr;
-        bool ok = new_event(&ev_start) && check(cudaEventRecord(ev_start, stream)) &&
-                  check(cudaStreamWaitEvent(dev->copy_in, ev_start, 0)) &&
-                  check(cudaMemcpy2DAsync(dB, pitch, B, ldb, K, N, cudaMemcpyHostToDevice, dev->copy_in)) &&
-                  new_event(&ev_b) && check(cudaEventRecord(ev_b, dev->copy_in)) &&
-                  check(cudaStreamWaitEvent(stream, ev_b, 0));
-        bool any_out = false;
-        for (int i = 0; i < chunks && ok; ++i) {
-            const long long r0 = i * rows_per;
-            const long long rows = (M - r0 < rows_per) ? M - r0 : rows_per;
-            char* a_i = dA + r0 * pitch;
-            int32_t* c_i = dC + r0 * ldc_dev;
-            cudaEvent_t ev_in = nullptr, ev_cmp = nullptr;
-            ok = check(cudaMemcpy2DAsync(a_i, pitch, static_cast<const char*>(A) + r0 * lda, lda, K, rows,
-                                         cudaMemcpyHostToDevice, dev->copy_in));
+        auto next_event = [&]() { return dev->host_events[n_ev++]; };
+        const long long rows_per = round_up((M + bi - 1) / bi, 256);
+        const long long cols_per = round_up((N + bj - 1) / bj, 256);
+        bi = static_cast<int>((M + rows_per - 1) / rows_per);
+        bj = static_cast<int>((N + cols_per - 1) / cols_per);
+        cudaEvent_t ev_a[kHostBlocks] = {}, ev_b[kHostBlocks] = {};
+        bool ok = true;
+        auto upload_a = [&](int i) {
+            const long long r0 = i * rows_per, rows = (M - r0 < rows_per) ? M - r0 : rows_per;
+            ok = ok && check(copy_rows(dA + r0 * pitch, pitch, static_cast<const char*>(A) + r0 * lda, lda, K, rows,
+                                       cudaMemcpyHostToDevice, dev->copy_in));
             if (ok && accumulate)
-                ok = check(cudaMemcpy2DAsync(c_i, ldc_dev * 4, C + r0 * ldc, ldc * 4, N * 4, rows,
-                                             cudaMemcpyHostToDevice, dev->copy_in));
-            ok = ok && new_event(&ev_in) && check(cudaEventRecord(ev_in, dev->copy_in)) &&
-                 check(cudaStreamWaitEvent(stream, ev_in, 0));
-            if (ok) {
-                const int gs = gemm_impl(a_unsigned, rows, N, K, a_i, pitch, reinterpret_cast<const int8_t*>(dB), pitch,
-                                         c_i, ldc_dev, accumulate, stream_v, 0);
-                if (gs != MIPGEMM_OK) { st = gs; ok = false; }
+                ok = check(copy_rows(dC + r0 * ldc_dev, ldc_dev * 4, C + r0 * ldc, ldc * 4, N * 4, rows,
+                                     cudaMemcpyHostToDevice, dev->copy_in));
+            ev_a[i] = next_event();
+            ok = ok && check(cudaEventRecord(ev_a[i], dev->copy_in));
+        };
+        auto upload_b = [&](int j) {
+            const long long c0 = j * cols_per, cols = (N - c0 < cols_per) ? N - c0 : cols_per;
+            ok = ok && check(copy_rows(dB + c0 * pitch, pitch, reinterpret_cast<const char*>(B) + c0 * ldb, ldb, K, cols,
+                                       cudaMemcpyHostToDevice, dev->copy_in));
+            ev_b[j] = next_event();
+            ok = ok && check(cudaEventRecord(ev_b[j], dev->copy_in));
+        };
+        cudaEvent_t ev_start = next_event();
+        ok = check(cudaEventRecord(ev_start, stream)) && check(cudaStreamWaitEvent(dev->copy_in, ev_start, 0)) &&
+             check(cudaStreamWaitEvent(dev->copy_out, ev_start, 0));
+        // upload order = order of first use by the row-major sweep over the blocks of C
+        if (ok) upload_a(0);
+        for (int j = 0; j < bj && ok; ++j) upload_b(j);
+        for (int i = 1; i < bi && ok; ++i) upload_a(i);
+        for (int i = 0; i < bi && ok; ++i) {
+            const long long r0 = i * rows_per, rows = (M - r0 < rows_per) ? M - r0 : rows_per;
+            ok = check(cudaStreamWaitEvent(stream, ev_a[i], 0));
+            for (int j = 0; j < bj && ok; ++j) {
+                const long long c0 = j * cols_per, cols = (N - c0 < cols_per) ? N - c0 : cols_per;
+                if (i == 0) ok = check(cudaStreamWaitEvent(stream, ev_b[j], 0));
+                if (!ok) break;
+                int32_t* c_ij = dC + r0 * ldc_dev + c0;
+                const int gs = gemm_impl(a_unsigned, rows, cols, K, dA + r0 * pitch, pitch,
+                                         reinterpret_cast<const int8_t*>(dB + c0 * pitch), pitch, c_ij, ldc_dev,
+                                         accumulate, stream_v, 0);
+                if (gs != MIPGEMM_OK) { st = gs; ok = false; break; }
+                cudaEvent_t ev_cmp = next_event();
+                ok = check(cudaEventRecord(ev_cmp, stream)) && check(cudaStreamWaitEvent(dev->copy_out, ev_cmp, 0)) &&
+                     check(copy_rows(C + r0 * ldc + c0, ldc * 4, c_ij, ldc_dev * 4, cols * 4, rows,
+                                     cudaMemcpyDeviceToHost, dev->copy_out));
             }
-            ok = ok && new_event(&ev_cmp) && check(cudaEventRecord(ev_cmp, stream)) &&
-                 check(cudaStreamWaitEvent(dev->copy_out, ev_cmp, 0)) &&
-                 check(cudaMemcpy2DAsync(C + r0 * ldc, ldc * 4, c_i, ldc_dev * 4, N * 4, rows, cudaMemcpyDeviceToHost,
-                                         dev->copy_out));
-            any_out = any_out || ok;
         }
-        // the caller's stream (and the release of the buffer) waits for both helper streams
-        if (new_event(&ev_done)) {
-            if (check(cudaEventRecord(ev_done, dev->copy_in))) check(cudaStreamWaitEvent(stream, ev_done, 0));
-        }
-        cudaEvent_t ev_out = nullptr;
-        if (any_out && new_event(&ev_out)) {
-            if (check(cudaEventRecord(ev_out, dev->copy_out))) check(cudaStreamWaitEvent(stream, ev_out, 0));
-        }
-        (void)cudaFreeAsync(base, stream);
+        // the caller's stream waits for both helper streams
+        cudaEvent_t ev_in_done = next_event(), ev_out_done = next_event();
+        if (check(cudaEventRecord(ev_in_done, dev->copy_in))) check(cudaStreamWaitEvent(stream, ev_in_done, 0));
+        if (check(cudaEventRecord(ev_out_done, dev->copy_out))) check(cudaStreamWaitEvent(stream, ev_out_done, 0));
         e = cudaStreamSynchronize(stream);
         if (st == MIPGEMM_OK && e != cudaSuccess) st = cuda_fail(e);
         if (st != MIPGEMM_OK) {   // make sure nothing of this call is still in flight
             (void)cudaStreamSynchronize(dev->copy_in);
             (void)cudaStreamSynchronize(dev->copy_out);
         }
-        for (int i = 0; i < n_ev; ++i) (void)cudaEventDestroy(ev[i]);
         return st;
     }
 
     if (K > 0) {
-        e = cudaMemcpy2DAsync(dA, pitch, A, lda, K, M, cudaMemcpyHostToDevice, stream);
-        if (e == cudaSuccess) e = cudaMemcpy2DAsync(dB, pitch, B, ldb, K, N, cudaMemcpyHostToDevice, stream);
-        if (e != cudaSuccess) st = cuda_fail(e);
+        check(copy_rows(dA, pitch, A, lda, K, M, cudaMemcpyHostToDevice, stream)) &&
+            check(copy_rows(dB, pitch, B, ldb, K, N, cudaMemcpyHostToDevice, stream));
     }
-    if (st == MIPGEMM_OK && accumulate) {
-        e = cudaMemcpy2DAsync(dC, ldc_dev * 4, C, ldc * 4, N * 4, M, cudaMemcpyHostToDevice, stream);
-        if (e != cudaSuccess) st = cuda_fail(e);
-    }
+    if (st == MIPGEMM_OK && accumulate)
+        check(copy_rows(dC, ldc_dev * 4, C, ldc * 4, N * 4, M, cudaMemcpyHostToDevice, stream));
     if (st == MIPGEMM_OK)
         st = gemm_impl(a_unsigned, M, N, K, dA, pitch, reinterpret_cast<const int8_t*>(dB), pitch, dC, ldc_dev,
                        accumulate, stream_v, 0);
-    if (st == MIPGEMM_OK) {
-        e = cudaMemcpy2DAsync(C, ldc * 4, dC, ldc_dev * 4, N * 4, M, cudaMemcpyDeviceToHost, stream);
-        if (e != cudaSuccess) st = cuda_fail(e);
-    }
-    (void)cudaFreeAsync(base, stream);
+    if (st == MIPGEMM_OK)
+        check(copy_rows(C, ldc * 4, dC, ldc_dev * 4, N * 4, M, cudaMemcpyDeviceToHost, stream));
     e = cudaStreamSynchronize(stream);
     if (st == MIPGEMM_OK && e != cudaSuccess) st = cuda_fail(e);
     return st;
@@ -948,6 +1200,7 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
                          int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
                          const uint8_t* X, const int8_t* Wt, int32_t* Y, int accumulate, void* stream_v) {
     tl_last_path = MIPGEMM_PATH_NONE;
+    const Tuning tun = tuning_now();
     ConvGeom g{Nb, H, W, Cin, Cout, 0, 0, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w};
     if (!conv_geometry(g)) return MIPGEMM_ERR_INVALID_ARG;
     const long long M = g.Nb * g.Ho * g.Wo;
@@ -968,31 +1221,56 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
     if (st != MIPGEMM_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
 
-    if (conv_tma_eligible(g, X, Wt) && g_tuning.force_path != MIPGEMM_PATH_IM2COL_EXPLICIT) {
+    if (conv_tma_eligible(g, X, Wt) && tun.force_path != MIPGEMM_PATH_IM2COL_EXPLICIT) {
         const int block_k = (Cin % 128 == 0) ? 128 : 64;
-        const Plan pl = make_plan(M, Cout, K, block_k, dev);
+        Plan pl;
         DenseParams p;
-        std::memset(&p, 0, sizeof(p));
-        fill_common(p, pl, M, Cout, Y, Cout, block_k, true, accumulate, dev);
-        p.a_im2col = 1;
-        p.conv_wo = static_cast<int>(g.Wo);
-        p.conv_howo = static_cast<int>(g.Ho * g.Wo);
-        p.conv_s = S;
-        p.c_chunks = static_cast<int>(Cin / block_k);
-        p.stride_w = stride_w; p.stride_h = stride_h;
-        p.pad_w = pad_w; p.pad_h = pad_h;
-        p.dil_w = dil_w; p.dil_h = dil_h;
-        if ((st = encode_im2col(&p.tmap_a, X, g, block_k, kBlockM)) != MIPGEMM_OK) return st;
-        if ((st = encode_tiled_2d(&p.tmap_b, Wt, K, Cout, K, block_k, pl.pair ? pl.block_n / 2 : pl.block_n)) !=
-            MIPGEMM_OK)
-            return st;
-        if ((st = run_dense(p, pl, M, Cout, Y, Cout, accumulate, dev, stream)) != MIPGEMM_OK) return st;
+        const bool cacheable = plan_cache_enabled();
+        PlanKey key;
+        bool hit = false;
+        if (cacheable) {
+            std::memset(&key, 0, sizeof(key));
+            auto pack2 = [](int a, int b) { return (static_cast<uint64_t>(static_cast<uint32_t>(a)) << 32) | static_cast<uint32_t>(b); };
+            const uint64_t words[] = {2, reinterpret_cast<uint64_t>(dev), g_tuning_epoch.load(std::memory_order_acquire),
+                                      accumulate ? 1u : 0u, out_mode_word(), static_cast<uint64_t>(Nb),
+                                      static_cast<uint64_t>(H), static_cast<uint64_t>(W), static_cast<uint64_t>(Cin),
+                                      static_cast<uint64_t>(Cout), pack2(R, S), pack2(stride_h, stride_w),
+                                      pack2(pad_h, pad_w), pack2(dil_h, dil_w), reinterpret_cast<uint64_t>(X),
+                                      reinterpret_cast<uint64_t>(Wt), reinterpret_cast<uint64_t>(Y)};
+            std::memcpy(key.w, words, sizeof(words));
+            hit = plan_lookup(key, &p, &pl);
+        }
+        if (hit) {
+            ++g_plan_hits;
+        } else {
+            pl = make_plan(M, Cout, K, block_k, dev);
+            std::memset(&p, 0, sizeof(p));
+            fill_common(p, pl, M, Cout, Y, Cout, block_k, true, accumulate, dev);
+            p.a_im2col = 1;
+            p.conv_wo = static_cast<int>(g.Wo);
+            p.conv_howo = static_cast<int>(g.Ho * g.Wo);
+            p.conv_s = S;
+            p.c_chunks = static_cast<int>(Cin / block_k);
+            p.stride_w = stride_w; p.stride_h = stride_h;
+            p.pad_w = pad_w; p.pad_h = pad_h;
+            p.dil_w = dil_w; p.dil_h = dil_h;
+            if ((st = encode_im2col(&p.tmap_a, X, g, block_k, kBlockM)) != MIPGEMM_OK) return st;
+            if ((st = encode_tiled_2d(&p.tmap_b, Wt, K, Cout, K, block_k, pl.pair ? pl.block_n / 2 : pl.block_n)) !=
+                MIPGEMM_OK)
+                return st;
+        }
+        if ((st = run_dense(p, pl, M, Cout, Y, Cout, accumulate, dev, stream, hit)) != MIPGEMM_OK) return st;
+        if (cacheable && !hit) {
+            ++g_plan_misses;
+            plan_store(key, p, pl);
+        }
         tl_last_path = (pl.pair ? MIPGEMM_PATH_DENSE_PAIR : MIPGEMM_PATH_DENSE) | MIPGEMM_PATH_IM2COL_TMA |
                        (pl.split_k > 1 ? MIPGEMM_PATH_SPLITK : 0);
+        if (log_enabled()) log_dense("conv (TMA im2col)", M, Cout, K, pl, p, hit);
         return MIPGEMM_OK;
     }
 
-    if (conv_gather_eligible(g) && g_tuning.force_path != MIPGEMM_PATH_IM2COL_EXPLICIT) {
+    if (conv_gather_eligible(g) && tun.force_path != MIPGEMM_PATH_IM2COL_EXPLICIT) {
         const int seg = S * static_cast<int>(Cin);
         const int slot = static_cast<int>(round_up(seg, 16));
         const long long Kp = static_cast<long long>(R) * slot;      // K with every filter row padded to its slot
@@ -1024,6 +1302,7 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
         if ((st = encode_tiled_2d(&p.tmap_b, wp, Kp, Cout, Kp, block_k, pl.block_n)) != MIPGEMM_OK) return st;
         if ((st = run_dense(p, pl, M, Cout, Y, Cout, accumulate, dev, stream)) != MIPGEMM_OK) return st;
         tl_last_path = MIPGEMM_PATH_DENSE | MIPGEMM_PATH_IM2COL_GATHER;
+        if (log_enabled()) log_dense("conv (gathered im2col)", M, Cout, Kp, pl, p, false);
         return MIPGEMM_OK;
     }
 
@@ -1040,6 +1319,9 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
     cudaError_t e = launch_im2col(ip, stream);
     ++g_launches;
     if (e != cudaSuccess) return cuda_fail(e);
+    if (log_enabled())
+        std::fprintf(stderr, "mipgemm: conv M=%lld N=%lld K=%lld -> explicit im2col matrix (pitch %lld), then:\n", M,
+                     static_cast<long long>(Cout), K, k_pitch);
     // The GEMM takes its own share (weight re-pitching when K % 16 != 0) from the same lease.
     return gemm_impl(true, M, Cout, K, cols, k_pitch, Wt, K, Y, Cout, accumulate, stream_v,
                      MIPGEMM_PATH_IM2COL_EXPLICIT, &scratch);
@@ -1052,15 +1334,19 @@ int mipgemm_device_status(void* stream_v) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     cudaError_t e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return cuda_fail(e);
-    unsigned int word = 0;
-    e = cudaMemcpy(&word, dev->status_word, sizeof(word), cudaMemcpyDeviceToHost);
-    if (e != cudaSuccess) return cuda_fail(e);
-    if (word != 0) {
-        e = cudaMemset(dev->status_word, 0, sizeof(word));
-        if (e != cudaSuccess) return cuda_fail(e);
-        return MIPGEMM_ERR_TIMEOUT;
+    st = take_status_word(dev->status_word);
+    // kernels launched by the allocation-free entry point report through a word of their own
+    int dev_index = 0;
+    unsigned int* static_word = nullptr;
+    if (cudaGetDevice(&dev_index) == cudaSuccess && dev_index >= 0 && dev_index < kMaxDevices) {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (g_noalloc[dev_index].ready) static_word = g_noalloc[dev_index].st.status_word;
     }
-    return MIPGEMM_OK;
+    if (static_word) {
+        const int st2 = take_status_word(static_word);
+        if (st == MIPGEMM_OK) st = st2;
+    }
+    return st;
 }
 
 int mipgemm_set_workspace(void* dev_ptr, size_t bytes) {
@@ -1182,6 +1468,26 @@ int mipgemm_gemm_ex(int a_unsigned, int b_unsigned, int a_order, int b_order, in
 
 uint64_t mipgemm_launch_count(void) { return g_launches.load(); }
 
+int mipgemm_release_staging(void) {
+    DeviceState* dev = nullptr;
+    int st = get_device(&dev);
+    if (st != MIPGEMM_OK) return st;
+    std::lock_guard<std::mutex> host_lock(dev->host_mutex);
+    if (dev->staging) {
+        cudaError_t e = cudaFree(dev->staging);
+        dev->staging = nullptr;
+        dev->staging_bytes = 0;
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return MIPGEMM_OK;
+}
+
+int mipgemm_plan_cache_stats(uint64_t* hits, uint64_t* misses) {
+    if (hits) *hits = g_plan_hits.load();
+    if (misses) *misses = g_plan_misses.load();
+    return plan_cache_enabled() ? 1 : 0;
+}
+
 int mipgemm_last_path(void) { return tl_last_path; }
 int mipgemm_last_cuda_error(void) { return tl_last_cuda_error; }
 
@@ -1221,13 +1527,41 @@ int mipgemm_set_weights_constant(int on) {
     return MIPGEMM_OK;
 }
 
+int mipgemm_register_constant_weights(const void* base, size_t bytes) {
+    if (!base || bytes == 0) return MIPGEMM_ERR_INVALID_ARG;
+    const uintptr_t lo = reinterpret_cast<uintptr_t>(base);
+    std::lock_guard<std::mutex> lock(g_ranges_mutex);
+    g_constant_ranges[lo] = lo + bytes;
+    g_constant_range_count.store(static_cast<int>(g_constant_ranges.size()), std::memory_order_release);
+    return MIPGEMM_OK;
+}
+
+int mipgemm_unregister_constant_weights(const void* base) {
+    std::lock_guard<std::mutex> lock(g_ranges_mutex);
+    if (g_constant_ranges.erase(reinterpret_cast<uintptr_t>(base)) == 0) return MIPGEMM_ERR_INVALID_ARG;
+    g_constant_range_count.store(static_cast<int>(g_constant_ranges.size()), std::memory_order_release);
+    return MIPGEMM_OK;
+}
+
+int mipgemm_debug_set(int flags, unsigned long long wait_budget_ns) {
+    if (flags & ~1) return MIPGEMM_ERR_INVALID_ARG;
+    g_debug_flags.store(flags);
+    g_wait_budget_ns.store(wait_budget_ns ? wait_budget_ns : 4000000000ull);
+    g_tuning_epoch.fetch_add(1, std::memory_order_acq_rel);   // cached launch parameters carry the old values
+    return MIPGEMM_OK;
+}
+
 int mipgemm_set_tuning(int block_n, int stages, int split_k, int force_path) {
     if (block_n != 0 && (block_n < 32 || block_n > 256 || block_n % 32 != 0)) return MIPGEMM_ERR_INVALID_ARG;
-    if (stages < 0 || stages > mip::kMaxStages || split_k < 0) return MIPGEMM_ERR_INVALID_ARG;
-    g_tuning.block_n = block_n;
-    g_tuning.stages = stages;
-    g_tuning.split_k = split_k;
-    g_tuning.force_path = force_path;
+    if (stages < 0 || stages > mip::kMaxStages || split_k < 0 || force_path < 0 || force_path > 0xFFFFFF)
+        return MIPGEMM_ERR_INVALID_ARG;
+    Tuning t;
+    t.block_n = block_n;
+    t.stages = stages;
+    t.split_k = split_k > 0xFFFF ? 0xFFFF : split_k;
+    t.force_path = force_path;
+    g_tuning_word.store(pack_tuning(t), std::memory_order_release);
+    g_tuning_epoch.fetch_add(1, std::memory_order_acq_rel);
     return MIPGEMM_OK;
 }
 
@@ -1243,24 +1577,12 @@ int mipgemm_set_tuning(int block_n, int stages, int split_k, int force_path) {
 // to another framework.  For them the re-pitching GEMM exists once more below with its
 // scratch in a fixed array that is part of the library image on every GPU that loads it.
 // Nothing on this path calls cudaMalloc, cudaMallocAsync, cudaFree or any other allocating
-// routine; it shares no state with the entry points above.
+// routine.  It shares the planner, the tensor-map encoders, the tuning overrides, the launch
+// counter and the per-thread last-path / last-error words with the entry points above, but
+// none of their device memory: its scratch and its status word are the two static symbols
+// defined near the top of this file.
 // ---------------------------------------------------------------------------------------
 namespace {
-
-// The scratch itself.  Host code must never use this name as an address: on the host it is
-// only a handle for cudaGetSymbolAddress (see noalloc_device()).
-static __device__ __align__(256) unsigned char g_static_scratch[MIPGEMM_STATIC_SCRATCH_BYTES];
-// Word that receives the "bounded wait expired" flag of kernels launched from this path.
-static __device__ unsigned int g_static_status;
-
-struct NoAllocDevice {
-    bool ready = false;
-    int status = MIPGEMM_OK;
-    DeviceState st;                 // sm_count, pair_clusters, status_word (-> g_static_status)
-    unsigned char* scratch = nullptr;   // device address of g_static_scratch on this device
-};
-NoAllocDevice g_noalloc[kMaxDevices];
-std::mutex g_noalloc_mutex;
 
 // Per-device set-up, done by the first call on each device with that device current:
 // capability check, tensor-map encoders, kernel attributes and the DEVICE addresses of the
@@ -1269,6 +1591,11 @@ int noalloc_device(NoAllocDevice** out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail(e);
+    thread_local int tl_context_bound = -1;      // (binds the device's context to this thread, see get_device())
+    if (tl_context_bound != dev) {
+        if ((e = cudaSetDevice(dev)) != cudaSuccess) return cuda_fail(e);
+        tl_context_bound = dev;
+    }
     if (dev < 0 || dev >= kMaxDevices) return MIPGEMM_ERR_UNSUPPORTED;
     std::lock_guard<std::mutex> lock(g_noalloc_mutex);
     NoAllocDevice& d = g_noalloc[dev];
@@ -1313,11 +1640,15 @@ int noalloc_device(NoAllocDevice** out) {
 extern "C" int mipgemm_s8s8s32_static_scratch(int64_t M, int64_t N, int64_t K, const int8_t* A, int64_t lda,
                                               const int8_t* B, int64_t ldb, int32_t* C, int64_t ldc,
                                               int accumulate, void* stream_v) {
+    tl_last_path = MIPGEMM_PATH_NONE;
     if (M < 0 || N < 0 || K < 0) return MIPGEMM_ERR_INVALID_ARG;
     if (M > 0x7FFFFF00LL || N > 0x7FFFFF00LL) return MIPGEMM_ERR_INVALID_ARG;
     if (lda < K || ldb < K || ldc < N) return MIPGEMM_ERR_INVALID_ARG;
     if (K > 131071) return MIPGEMM_ERR_K_TOO_LARGE;
-    if (M == 0 || N == 0) return MIPGEMM_OK;
+    if (M == 0 || N == 0) {
+        tl_last_path = MIPGEMM_PATH_TRIVIAL;
+        return MIPGEMM_OK;
+    }
     if (!C || reinterpret_cast<uintptr_t>(C) % 4 != 0) return MIPGEMM_ERR_INVALID_ARG;
     if (K > 0 && (!A || !B)) return MIPGEMM_ERR_INVALID_ARG;
     // How much of the static array this call needs; refuse before anything is enqueued.
@@ -1334,6 +1665,7 @@ extern "C" int mipgemm_s8s8s32_static_scratch(int64_t M, int64_t N, int64_t K, c
             if ((e = launch_fill_zero(C, ldc, M, N, stream)) != cudaSuccess) return cuda_fail(e);
             ++g_launches;
         }
+        tl_last_path = MIPGEMM_PATH_TRIVIAL;
         return MIPGEMM_OK;
     }
 
@@ -1345,6 +1677,7 @@ extern "C" int mipgemm_s8s8s32_static_scratch(int64_t M, int64_t N, int64_t K, c
     const void* b_use = B;
     long long lda_use = lda, ldb_use = ldb;
     size_t used = 0;
+    int flags = 0;
     if (!aligned16(A, lda)) {
         unsigned char* dst = nd->scratch + used;
         used += align256(static_cast<size_t>(M) * pitch);
@@ -1352,6 +1685,7 @@ extern "C" int mipgemm_s8s8s32_static_scratch(int64_t M, int64_t N, int64_t K, c
         ++g_launches;
         a_use = dst;
         lda_use = pitch;
+        flags |= MIPGEMM_PATH_REPACK;
     }
     if (!aligned16(B, ldb)) {
         unsigned char* dst = nd->scratch + used;
@@ -1360,6 +1694,7 @@ extern "C" int mipgemm_s8s8s32_static_scratch(int64_t M, int64_t N, int64_t K, c
         ++g_launches;
         b_use = dst;
         ldb_use = pitch;
+        flags |= MIPGEMM_PATH_REPACK;
     }
 
     const int block_k = 128;
@@ -1371,5 +1706,19 @@ extern "C" int mipgemm_s8s8s32_static_scratch(int64_t M, int64_t N, int64_t K, c
     if ((st = encode_tiled_2d(&p.tmap_b, b_use, K, N, ldb_use, block_k, pl.pair ? pl.block_n / 2 : pl.block_n)) !=
         MIPGEMM_OK)
         return st;
-    return run_dense(p, pl, M, N, C, ldc, accumulate, &nd->st, stream);
+    if ((st = run_dense(p, pl, M, N, C, ldc, accumulate, &nd->st, stream)) != MIPGEMM_OK) return st;
+    if (pl.split_k > 1) flags |= MIPGEMM_PATH_SPLITK;
+    tl_last_path = (pl.pair ? MIPGEMM_PATH_DENSE_PAIR : MIPGEMM_PATH_DENSE) | flags;
+    return MIPGEMM_OK;
+}
+
+// Allocation-free status query for the entry point above: waits for `stream`, then reads and clears
+// the static status word (plain copies from and to the symbol's address; nothing is allocated).
+extern "C" int mipgemm_static_scratch_status(void* stream_v) {
+    NoAllocDevice* nd = nullptr;
+    int st = noalloc_device(&nd);
+    if (st != MIPGEMM_OK) return st;
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream_v));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return take_status_word(nd->st.status_word);
 }

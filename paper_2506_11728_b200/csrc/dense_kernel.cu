@@ -55,8 +55,9 @@ __device__ __forceinline__ TileCoord decode_unit(const DenseParams& p, int unit,
     const int first_n = g * p.group_n;
     const int gsize = min(p.group_n, p.tiles_n - first_n);
     const int r = t - g * per_group;
-    const int tm = r / gsize;
+    int tm = r / gsize;
     const int tn = first_n + (r - tm * gsize);
+    if ((p.raster & 1) && (g & 1)) tm = p.tiles_m - 1 - tm;   // serpentine: the A slabs at the turn are still in L2
     TileCoord c;
     c.m0 = tm * rows_per_tile;
     c.n0 = tn * p.block_n;
@@ -196,6 +197,7 @@ __device__ __forceinline__ void tma_store_slab(const DenseParams& p, uint32_t bu
 #endif
     if (issuer && elect_one()) {
         if (p.batch > 1) tma_store_3d(&p.tmap_c, buf, x, y, z);
+        else if (p.c_evict_first) tma_store_2d_hint(&p.tmap_c, buf, x, y, l2_policy_evict_first());
         else tma_store_2d(&p.tmap_c, buf, x, y);
         tma_store_commit();
     }
@@ -429,10 +431,11 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 
     const int total_units = p.tiles_m * p.tiles_n * p.split_k * (p.batch > 1 ? p.batch : 1);
     const uint64_t budget = p.wait_budget_ns;
+    uint32_t issued = 0;   // producer warp: k-blocks whose loads have been issued (the unwinding path needs it)
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (whole warp loops)
-        uint32_t s = 0, phase = 0, issued = 0;
+        uint32_t s = 0, phase = 0;
         bool ok = true;
         const uint32_t tx_bytes = kGather ? b_bytes : (kPair ? 2u * stage_bytes : stage_bytes);
         for (int unit = first_unit; unit < total_units && ok; unit += unit_stride) {
@@ -510,21 +513,6 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
             }
         }
-        if (!ok && leader) {
-            // Unwinding: wait (bounded) until every copy already issued has landed.  (A peer
-            // CTA cannot observe its copies -- they complete on the leader's barrier; it is
-            // held by the final cluster barrier until the leader has finished unwinding.)
-            const uint32_t n = min(issued, static_cast<uint32_t>(p.stages));
-            for (uint32_t i = 1; i <= n; ++i) {
-                const uint32_t idx = issued - i;
-                const uint32_t st = idx % p.stages;
-                const uint32_t ph = (idx / p.stages) & 1u;
-                const uint64_t t0 = globaltimer_ns();
-                while (!mbar_try_wait(bar_full + 8u * st, ph)) {
-                    if (globaltimer_ns() - t0 > budget) break;
-                }
-            }
-        }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (whole warp loops)
         if (leader) {
@@ -567,7 +555,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
                 }
                 if (t == 0) MIP_STAMP(4);
-                if (ok) {
+                if (ok && !(p.debug_flags & 1)) {   // (test hook, bit 0: the "accumulator ready" signal is withheld)
                     const uint32_t tfull_local = bar_tfull + 8u * acc;
                     const uint32_t tfull_peer = kPair ? mapa_u32(tfull_local, 1) : 0u;
                     if (elect_one()) {
@@ -578,16 +566,6 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                             mma_commit(tfull_local);
                         }
                     }
-                }
-            }
-            if (!ok) {
-                // Unwinding: let every MMA already issued retire before TMEM is released.
-                if (elect_one()) {
-                    if (kPair) mma_commit_pair(bar_drain); else mma_commit(bar_drain);
-                }
-                const uint64_t t0 = globaltimer_ns();
-                while (!mbar_try_wait(bar_drain, 0)) {
-                    if (globaltimer_ns() - t0 > budget) break;
                 }
             }
         }
@@ -735,7 +713,11 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 #ifdef MIPGEMM_TRACE
             const long long tt0 = clock64();
 #endif
-            if (!mbar_wait(bar_tfull + 8u * acc, acc_phase, abort_flag, budget)) break;
+            bool gave_up = !mbar_wait(bar_tfull + 8u * acc, acc_phase, abort_flag, budget);
+            // Each warp waits on its own clock, but slab stores meet at named barriers: the four warps decide
+            // together whether to go on, so none can leave while another still expects it there.
+            if (p.c_mode == 1 && p.cluster_split <= 1) gave_up = named_bar_or(1, 128, gave_up);
+            if (gave_up) break;
 #ifdef MIPGEMM_TRACE
             if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { p.trace[59] += clock64() - tt0; p.trace[60] += 1; }
 #endif
@@ -903,6 +885,38 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 
     tc_fence_before();
     __syncthreads();
+    if (*abort_flag != 0) {
+        // Unwinding (uniform: every role has left its loop, so nobody writes the flag any more).  Some role gave
+        // up a wait; whatever is still on its way to this CTA must arrive before shared and tensor memory are
+        // given back, whichever role it was that gave up:
+        //  * the producer warp waits (bounded) until the copies of the last `stages` k-blocks it issued have
+        //    landed (a peer CTA cannot observe its own copies -- they complete on the leader's barrier; it is
+        //    held by the cluster barrier below until the leader has finished here);
+        //  * the MMA warp lets every MMA it issued retire (one more commit, bounded wait).
+        if (warp == 0 && leader) {
+            const uint32_t n = min(issued, static_cast<uint32_t>(p.stages));
+            for (uint32_t i = 1; i <= n; ++i) {
+                const uint32_t idx = issued - i;
+                const uint32_t st = idx % p.stages;
+                const uint32_t ph = (idx / p.stages) & 1u;
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(bar_full + 8u * st, ph)) {
+                    if (globaltimer_ns() - t0 > budget) break;
+                }
+            }
+        }
+        if (warp == 1 && leader) {
+            if (elect_one()) {
+                if (kPair) mma_commit_pair(bar_drain); else mma_commit(bar_drain);
+            }
+            const uint64_t t0 = globaltimer_ns();
+            while (!mbar_try_wait(bar_drain, 0)) {
+                if (globaltimer_ns() - t0 > budget) break;
+            }
+            tc_fence_before();
+        }
+        __syncthreads();
+    }
     if (threadIdx.x == 0) MIP_STAMP(8);
     if (kPair) {   // neither CTA may leave while the other can still reach its shared memory
         cluster_arrive();

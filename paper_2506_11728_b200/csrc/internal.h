@@ -15,6 +15,22 @@ inline int pdl_allowed() {
     return v;
 }
 
+// Integer environment variable read once per name (experiment switches; `fallback` when unset).
+inline int env_int(const char* name, int fallback) {
+    const char* e = std::getenv(name);
+    return e ? std::atoi(e) : fallback;
+}
+
+// Experiment switch: read once, or on every call when MIPGEMM_LIVE_ENV=1 (A/B runs inside one process;
+// cached plans are bypassed then).
+inline bool live_env() {
+    static const bool v = env_int("MIPGEMM_LIVE_ENV", 0) != 0;
+    return v;
+}
+#define MIP_ENV_KNOB(name, fallback) \
+    ([]() -> int { static const int cached = ::mip::env_int(name, fallback); \
+                   return ::mip::live_env() ? ::mip::env_int(name, fallback) : cached; }())
+
 constexpr int kBlockM = 128;          // rows of C per CTA (TMEM lanes)
 constexpr int kDenseThreads = 192;    // producer warp, MMA warp, 4 epilogue warps
 constexpr int kDenseQ8Threads = 320;  // 8-bit-code epilogue: 8 epilogue warps
@@ -51,6 +67,8 @@ struct alignas(64) DenseParams {
     long long stride_c;      // elements between consecutive C matrices of a batch
     int cluster_split;       // > 1: the split_k CTAs sharing a tile form a cluster and reduce through DSMEM
     int group_n;             // n-tiles per rasterisation group
+    int raster;              // bit 0: serpentine (odd groups are swept bottom to top)
+    int c_evict_first;       // 1: TMA tile stores of C carry an evict-first L2 hint
     int accumulate;          // epilogue adds the incoming C
     int use_red;             // epilogue reduces with red.global.add (split-K)
     int store_vec;           // 8, 4 or 1 int32 per store instruction
@@ -80,6 +98,7 @@ struct alignas(64) DenseParams {
     int g_chunks;            // 16-byte chunks per row of A (R * g_slot / 16)
     unsigned int* status;    // device word, bit 0 set when a bounded wait expired
     unsigned long long wait_budget_ns;
+    int debug_flags;         // test hook (mipgemm_debug_set): bit 0 = never signal "accumulator ready"
     unsigned long long* trace;   // timeline stamps of CTA 0; only read by builds with -DMIPGEMM_TRACE
 };
 
@@ -115,6 +134,7 @@ struct alignas(64) SkinnyRingParams {
     int slots, tokens_in_smem;   // filled in by the launcher
     unsigned int* status;
     unsigned long long wait_budget_ns;
+    int debug_flags;             // test hook (mipgemm_debug_set): bit 0 = the first CTA never loads its second chunk
 };
 bool skinny_ring_supported(const SkinnyParams& p, int sm_count);
 cudaError_t skinny_ring_init();  // once per device

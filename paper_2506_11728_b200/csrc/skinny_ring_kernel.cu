@@ -146,7 +146,10 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
         for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
             for (int ch = 0; ch < chunks; ++ch) {
                 if (!mbar_wait(bar_empty + 8u * s, phase ^ 1u, abort_flag, budget)) { ok = false; break; }
-                if (elect_one()) {
+                // (test hook, bit 0: CTA 0 leaves out the second chunk of its first unit, so its consumers' wait
+                // for that slot runs out)
+                const bool withheld = (p.debug_flags & 1) && blockIdx.x == 0 && u == 0 && ch == 1;
+                if (elect_one() && !withheld) {
                     mbar_arrive_expect_tx(bar_full + 8u * s, kSlotBytes);
                     tma_load_3d(ring + s * kSlotBytes, &p.tmap_b, bar_full + 8u * s, 0, u * 16, ch * 8);
                 }
@@ -185,6 +188,10 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
             }
             ok = mbar_wait(bar_tokens, 0u, abort_flag, budget);
         }
+        // Every consumer thread waits on its own clock, but the warps meet at named barriers once per unit:
+        // whether to go on is decided by all 256 together (here and at the end of every unit), so that no warp
+        // can leave while another still expects it at a barrier.
+        ok = !named_bar_or(1, 256, !ok);
         TokenRegs cur = {}, nxt;
         if (ok) {
             if (tsm) load_tokens_smem<kSecondTokenBlock>(cur, sx0, sx1, warp, p.K, t, tok0_ok, tok1_ok);
@@ -221,7 +228,7 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
                 cur = nxt;
                 if (++s == static_cast<uint32_t>(kRingSlots)) { s = 0; phase ^= 1u; }
             }
-            if (!ok) break;
+            // (a warp that gave up still brings its partials -- garbage then -- to the barrier below)
             // accumulator fragment: d0 (row g, col 2t), d1 (g, 2t+1), d2 (g+8, 2t), d3 (g+8, 2t+1);
             // row = weight row of the unit, col = token
             red[warp][g][2 * t] = acc0[0];
@@ -234,7 +241,7 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
                 red[warp][g + 8][8 + 2 * t] = acc1[2];
                 red[warp][g + 8][8 + 2 * t + 1] = acc1[3];
             }
-            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (named_bar_or(1, 256, !ok)) { ok = false; break; }   // partials are in place -- or somebody gave up
             const long long col = static_cast<long long>(u) * 16 + n;
             if (tok < p.M && (kSecondTokenBlock || tok < 8) && col < p.N) {
                 int sum = 0;
@@ -289,14 +296,16 @@ cudaError_t launch_ring_t(SkinnyRingParams p, int grid, cudaStream_t stream) {
         // promise, while the previous call drains) the other keeps streaming, and it no longer matters
         // which call's CTAs the block scheduler puts side by side.  Measured over a chain of 264 decode
         // GEMMs: 2.49 -> 2.28 ms without the promise, 2.06 -> 1.96 ms with it.
-        const int fit_min = 2;
+        const int fit_min = MIP_ENV_KNOB("MIPGEMM_RING_FIT_MIN", 2);
+        const int const_grid = MIP_ENV_KNOB("MIPGEMM_RING_CONST_GRID", 0);
         const int budget = 228 * 1024 / 2 - 2048;
         const int fit = (budget - fixed - tok_bytes) / kSlotBytes;
         if (fit >= fit_min) {
             p.tokens_in_smem = 1;
             slots = fit < kMaxRingSlots ? fit : kMaxRingSlots;
             const int units = (p.N + 15) / 16;
-            grid = units < 2 * grid ? units : 2 * grid;
+            const int cap = (const_grid && p.b_constant) ? grid : 2 * grid;
+            grid = units < cap ? units : cap;
         }
     }
     p.slots = slots;

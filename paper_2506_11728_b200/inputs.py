@@ -12,6 +12,9 @@ same shapes, plausible value distributions, no dataset needed.
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 
 _GOLDEN = np.uint64(0x9E3779B97F4A7C15)
@@ -31,58 +34,63 @@ def _mix64(idx: np.ndarray, seed: int) -> np.ndarray:
     return z
 
 
-def _chunks(count: int, start: int = 0):
-    pos = 0
-    while pos < count:
+def _fill(out: np.ndarray, convert, start: int = 0) -> np.ndarray:
+    """out[i] = convert(hash words of element indices start+i), chunk by chunk.  Every element is a
+    pure function of its own index, so large arrays are filled by a few threads at once (NumPy
+    releases the interpreter lock inside its loops) with the same result as a serial fill."""
+    count = out.size
+
+    def one(pos: int) -> None:
         n = min(_CHUNK, count - pos)
-        yield pos, np.arange(start + pos, start + pos + n, dtype=np.uint64)
-        pos += n
+        out[pos:pos + n] = convert(np.arange(start + pos, start + pos + n, dtype=np.uint64))
+
+    starts = range(0, count, _CHUNK)
+    workers = min(len(starts), _THREADS)
+    if workers <= 1:
+        for pos in starts:
+            one(pos)
+    else:
+        with ThreadPoolExecutor(max_workers=workers) as pool:
+            list(pool.map(one, starts))
+    return out
+
+
+_THREADS = max(1, min(16, os.cpu_count() or 1))
 
 
 def raw_u64(count: int, seed: int, start: int = 0) -> np.ndarray:
     """``count`` 64-bit hash words for element indices start .. start+count-1."""
-    out = np.empty(count, dtype=np.uint64)
-    for pos, idx in _chunks(count, start):
-        out[pos:pos + idx.size] = _mix64(idx, seed)
-    return out
+    return _fill(np.empty(count, dtype=np.uint64), lambda idx: _mix64(idx, seed), start)
 
 
 def uniform_s8(count: int, seed: int) -> np.ndarray:
     """int8 uniform over [-128, 127]."""
-    out = np.empty(count, dtype=np.int8)
-    for pos, idx in _chunks(count):
-        out[pos:pos + idx.size] = (_mix64(idx, seed) & np.uint64(0xFF)).astype(np.uint8).view(np.int8)
-    return out
+    return _fill(np.empty(count, dtype=np.int8),
+                 lambda idx: (_mix64(idx, seed) & np.uint64(0xFF)).astype(np.uint8).view(np.int8))
 
 
 def uniform_u8(count: int, seed: int) -> np.ndarray:
     """uint8 uniform over [0, 255] (post-ReLU activations)."""
-    out = np.empty(count, dtype=np.uint8)
-    for pos, idx in _chunks(count):
-        out[pos:pos + idx.size] = (_mix64(idx, seed) & np.uint64(0xFF)).astype(np.uint8)
-    return out
+    return _fill(np.empty(count, dtype=np.uint8), lambda idx: (_mix64(idx, seed) & np.uint64(0xFF)).astype(np.uint8))
 
 
 def normal_s8(count: int, seed: int, sigma: float, lo: int = -128, hi: int = 127) -> np.ndarray:
     """int8 values round(sigma * z), z standard normal (Box-Muller on the two
     32-bit halves of the hash word), clipped to [lo, hi]."""
-    out = np.empty(count, dtype=np.int8)
-    for pos, idx in _chunks(count):
+    def convert(idx):
         h = _mix64(idx, seed)
         u1 = ((h >> np.uint64(32)).astype(np.float64) + 1.0) / 4294967296.0
         u2 = (h & np.uint64(0xFFFFFFFF)).astype(np.float64) / 4294967296.0
         z = np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
-        out[pos:pos + idx.size] = np.clip(np.rint(sigma * z), lo, hi).astype(np.int8)
-    return out
+        return np.clip(np.rint(sigma * z), lo, hi).astype(np.int8)
+    return _fill(np.empty(count, dtype=np.int8), convert)
 
 
 def uniform_s32(count: int, seed: int, bound: int = 1 << 20) -> np.ndarray:
     """int32 uniform over [-bound, bound] (seeded C for accumulate=1 runs)."""
-    out = np.empty(count, dtype=np.int32)
     span = np.uint64(2 * bound + 1)
-    for pos, idx in _chunks(count):
-        out[pos:pos + idx.size] = ((_mix64(idx, seed) >> np.uint64(11)) % span).astype(np.int64) - bound
-    return out
+    return _fill(np.empty(count, dtype=np.int32),
+                 lambda idx: ((_mix64(idx, seed) >> np.uint64(11)) % span).astype(np.int64) - bound)
 
 
 def seed_for(config_index: int, operand_id: int) -> int:

@@ -87,3 +87,15 @@ def test_tuning_validation(mg):
         mg.mipgemm_set_tuning(block_n=48)
     mg.mipgemm_set_tuning(block_n=128, stages=3)
     mg.mipgemm_set_tuning()
+
+
+def test_constant_weight_ranges_are_bookkeeping_only(mg):
+    """Registering and unregistering weight ranges touches no device."""
+    assert mg.mipgemm_register_constant_weights(0, 16, check=False) == mg.ERR_INVALID_ARG
+    assert mg.mipgemm_register_constant_weights(4096, 0, check=False) == mg.ERR_INVALID_ARG
+    assert mg.mipgemm_register_constant_weights(4096, 1 << 20) == mg.OK
+    assert mg.mipgemm_register_constant_weights(1 << 30, 1 << 20) == mg.OK
+    assert mg.mipgemm_unregister_constant_weights(8192, check=False) == mg.ERR_INVALID_ARG   # not a base
+    assert mg.mipgemm_unregister_constant_weights(4096) == mg.OK
+    assert mg.mipgemm_unregister_constant_weights(4096, check=False) == mg.ERR_INVALID_ARG   # already gone
+    assert mg.mipgemm_unregister_constant_weights(1 << 30) == mg.OK

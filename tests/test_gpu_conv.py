@@ -155,7 +155,7 @@ def test_resnet50_layers_batch2_full(mg, layer):
     check_conv(mg, 2, H, W, Cin, Cout, R, S, (st, st), (pd, pd), seed=inputs.seed_for(3, layer))
 
 
-@pytest.mark.parametrize("layer", [0, 2, 6, 8, 16, 18, 22])
+@pytest.mark.parametrize("layer", range(len(inputs.RESNET50_CONVS)))
 def test_resnet50_layers_batch32_sampled_images(mg, layer):
     """Full batch on the GPU; the oracle recomputes two whole images (the output of image n
     depends on image n only) -- first and last, so tile runs that cross image borders count."""
@@ -180,7 +180,25 @@ def test_implicit_im2col_cta_pair(mg, case):
         mg.mipgemm_set_tuning()
 
 
-@pytest.mark.parametrize("layer", [0, 6, 14, 22])
+@pytest.mark.parametrize("layer", [12, 16, 18, 22])
+def test_resnet50_k_heavy_layers_batch32_cta_pair(mg, layer):
+    """The K >= 2304 layers once more with the CTA-pair kernel forced (im2col loads in their cta_group::2
+    form at full size): three whole images against the oracle."""
+    _cnt, H, W, Cin, Cout, R, S, st, pd = inputs.RESNET50_CONVS[layer]
+    Nb = 32
+    X, Wt = conv_inputs(Nb, H, W, Cin, Cout, R, S, inputs.seed_for(3, layer) + 3)
+    mg.mipgemm_set_tuning(force_path=mg.PATH_DENSE_PAIR)
+    try:
+        got, path = run_conv(mg, X, Wt, (st, st), (pd, pd), (1, 1))
+    finally:
+        mg.mipgemm_set_tuning()
+    assert path & mg.PATH_MASK == mg.PATH_DENSE_PAIR and path & mg.PATH_IM2COL_TMA
+    for n in (0, 13, Nb - 1):
+        want = orc.conv(X[n:n + 1], Wt, stride=(st, st), pad=(pd, pd))
+        assert np.array_equal(got[n:n + 1], want), "image %d: %s" % (n, first_mismatch(got[n:n + 1], want))
+
+
+@pytest.mark.parametrize("layer", range(len(inputs.RESNET50_CONVS)))
 def test_resnet50_layers_batch128_sampled_images(mg, layer):
     """Batch 128 (the largest configuration: the stem's GEMM has 1.6 M rows): full batch on the GPU,
     three whole images recomputed by the oracle."""

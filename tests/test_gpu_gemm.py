@@ -208,6 +208,41 @@ def test_skinny_with_constant_weights_promise(mg):
         mg.mipgemm_set_weights_constant(0)
 
 
+def test_skinny_with_registered_weight_ranges(mg):
+    """The per-buffer form of the promise: calls whose B lies inside a registered range fetch it early, other
+    calls do not; results are the oracle's either way, also when the tokens are the previous call's output."""
+    import torch
+    M, N, K = 4, 4096, 4096
+    A0 = inputs.uniform_s8(M * K, 5100)
+    B1 = inputs.uniform_s8(N * K, 5200)
+    B2 = inputs.uniform_s8(N * 4 * N, 5300)
+    dA0, _k0 = to_dev(A0)
+    dB1, _k1 = to_dev(B1)
+    dB2, _k2 = to_dev(B2)
+    dC = [torch.full((M * N,), 0x7F7F7F7F, dtype=torch.int32, device="cuda") for _ in range(4)]
+    mg.mipgemm_register_constant_weights(dB1)                      # whole tensor
+    mg.mipgemm_register_constant_weights(dB2, dB2.numel() // 2)    # only the first half: B2 is NOT covered
+    try:
+        torch.cuda.synchronize()
+        mg.mipgemm_s8s8s32(M, N, K, dA0, K, dB1, K, dC[0], N, False)
+        assert mg.mipgemm_last_path() & mg.PATH_MASK == mg.PATH_SKINNY
+        mg.mipgemm_s8s8s32(M, N, 4 * N, dC[0].view(torch.uint8), 4 * N, dB2, 4 * N, dC[1], N, False)
+        mg.mipgemm_s8s8s32(M, N, K, dC[1].view(torch.uint8)[:M * K], K, dB1, K, dC[2], N, False)
+        mg.mipgemm_s8s8s32(M, N, K, dC[2].view(torch.uint8)[:M * K], K, dB1, K, dC[3], N, False)
+        torch.cuda.synchronize()
+        assert mg.mipgemm_device_status() == mg.OK
+    finally:
+        mg.mipgemm_unregister_constant_weights(dB1)
+        mg.mipgemm_unregister_constant_weights(dB2)
+    w0 = orc.gemm(A0, B1, M, N, K)
+    w1 = orc.gemm(w0.view(np.int8), B2, M, N, 4 * N)
+    w2 = orc.gemm(w1.view(np.int8)[:M * K].copy(), B1, M, N, K)
+    w3 = orc.gemm(w2.view(np.int8)[:M * K].copy(), B1, M, N, K)
+    for d, want in enumerate([w0, w1, w2, w3]):
+        got = dC[d].cpu().numpy()
+        assert np.array_equal(got, want), "launch %d: %s" % (d, first_mismatch(got, want))
+
+
 @pytest.mark.parametrize("promise", [0, 1])
 def test_skinny_ring_slots_reused_with_two_ctas_per_sm(mg, promise):
     """Few ring slots, several chunks per CTA and two CTAs streaming on every SM: a slot is refilled (an

@@ -1,11 +1,11 @@
-"""Full-size members of the square sweep: sampled rows / tiles against the oracle and
-whole-matrix checksum identities (exact in int64), on the GPU's complete output."""
+"""Full-size members of the square sweep: the whole result against the oracle up to 8192^3, sampled rows,
+columns and tiles above, and whole-matrix checksum identities (exact in int64) on the GPU's complete output."""
 import numpy as np
 import pytest
 
 from oracle import mip_oracle as orc
 from paper_2506_11728_b200 import inputs
-from gpu_util import run_gemm
+from gpu_util import first_mismatch, run_gemm
 
 pytestmark = pytest.mark.gpu
 
@@ -73,7 +73,11 @@ def test_square_sweep_large_members(mg, n):
     B = inputs.uniform_s8(n * n, inputs.seed_for(2, n) + 2)
     C, path = run_gemm(mg, "s8", n, n, n, A, B)
     assert path & mg.PATH_MASK in (mg.PATH_DENSE, mg.PATH_DENSE_PAIR)
-    sampled_parity(A, B, C, n, n, n, rng)
+    if n <= 8192:       # the whole matrix against the oracle (seconds of CPU time up to this size)
+        want = orc.gemm(A, B, n, n, n)
+        assert np.array_equal(C, want), first_mismatch(C.reshape(n, n), want.reshape(n, n))
+    else:               # above that: sampled rows, columns and tiles, exactly
+        sampled_parity(A, B, C, n, n, n, rng)
     checksum_identities(A, B, C, n, n, n, rng)
 
 

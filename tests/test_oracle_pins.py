@@ -57,7 +57,7 @@ def _rand_case(rng, M, N, K, a_unsigned):
 @pytest.mark.parametrize("accumulate", [0, 1])
 def test_p1_brute_force_all_tiny_shapes(a_unsigned, accumulate):
     rng = np.random.default_rng(1234 + 2 * a_unsigned + accumulate)
-    shapes = [(m, n, k) for m in range(1, 6) for n in range(1, 6) for k in range(1, 6)]
+    shapes = [(m, n, k) for m in range(1, 10) for n in range(1, 10) for k in range(1, 10)]
     shapes += [tuple(int(v) for v in rng.integers(1, 34, size=3)) for _ in range(12)]
     for (M, N, K) in shapes:
         A, lda, B, ldb, C, ldc = _rand_case(rng, M, N, K, a_unsigned)

@@ -5,7 +5,9 @@ memory-planned runtime that owns the device, a real-time loop, a plug-in under a
 framework's pool): its re-pitching scratch is a fixed array inside the library instead of a
 cudaMallocAsync allocation.  The array is shared by every call and keeps the previous call's
 bytes, so the test makes two different calls in a row and compares each, bit for bit, with what
-``mipgemm_s8s8s32`` produces for the same operands.  This file is collected last on purpose: if
+``mipgemm_s8s8s32`` produces for the same operands and with the CPU oracle; after each call the
+entry point's own allocation-free status query must report that no device-side wait ran out, and
+the path query must name the kernel family that ran.  This file is collected last on purpose: if
 it fails, a run that stops at the first failure has already run everything else; it also passes
 when it is the only test of a fresh process (the new entry point does its own device set-up).
 """
@@ -36,8 +38,18 @@ def _both(mg, M, N, K, lda, ldb, ldc, accumulate, seed, misalign=0):
     for fn in (mg.mipgemm_s8s8s32_static_scratch, mg.mipgemm_s8s8s32):
         dC, _kc = to_dev(C0)
         fn(M, N, K, dA, lda, dB, ldb, dC, ldc, accumulate)
+        if fn is mg.mipgemm_s8s8s32_static_scratch:
+            assert mg.mipgemm_static_scratch_status() == mg.OK       # synchronises; nothing gave up a wait
+            path = mg.mipgemm_last_path()
+            assert path & mg.PATH_MASK in (mg.PATH_DENSE, mg.PATH_DENSE_PAIR), hex(path)
+            needs_scratch = mg.mipgemm_workspace_query_gemm(M, N, K, dA, lda, dB, ldb, dC, ldc) > 0
+            assert bool(path & mg.PATH_REPACK) == needs_scratch
         torch.cuda.synchronize()
         outs.append(dC.cpu().numpy().view(np.int32).copy())
+    # the oracle's word on the same operands (padding columns of C keep their seeded contents)
+    from oracle import mip_oracle as orc
+    want = orc.gemm(A, B, M, N, K, lda=lda, ldb=ldb, C=C0.copy(), ldc=ldc, accumulate=bool(accumulate))
+    assert np.array_equal(outs[0], want)
     return outs
 
 
