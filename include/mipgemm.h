@@ -237,7 +237,7 @@ int mipgemm_conv_u8s8f32_dequant(int64_t Nb, int64_t H, int64_t W, int64_t Cin, 
  * staging buffer, runs the device entry point, copies the M x N result back into C (padding
  * columns of the host C are left untouched; with accumulate != 0 the host C is uploaded
  * first) and SYNCHRONISES the stream before returning.  Large problems (>= 32 MB) are cut into
- * up to 8 x 8 blocks of C that three streams pipeline -- operand blocks in, compute on
+ * up to 4 x 4 blocks of C that three streams pipeline -- operand blocks in, compute on
  * `stream`, finished blocks out -- so both directions of the host link are busy at once; pinned
  * host memory is what makes those copies asynchronous.  The staging buffer (one per device, as
  * large as the largest call so far) stays allocated between calls; mipgemm_release_staging()

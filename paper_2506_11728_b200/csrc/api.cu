@@ -564,7 +564,8 @@ int run_dense(DenseParams& p, const Plan& pl, long long M, long long N, int32_t*
     const long long units = static_cast<long long>(pl.tiles_m) * pl.tiles_n * pl.split_k;
     const int b_rows = pl.pair ? pl.block_n / 2 : pl.block_n;
     const size_t smem = static_cast<size_t>(pl.stages) * (kBlockM * p.block_k + b_rows * p.block_k) +
-                        kStagingBytes + kCtrlBytes + 1024;
+                        kStagingBytes + kCtrlBytes + 1024 +
+                        (p.g_staged ? 64 + 2 * static_cast<size_t>(p.g_rowbuf_stride) + p.g_table_bytes : 0);
     if ((p.c_mode == 1 || p.c_mode == 2) && !c_map_ready) {
         cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(M)};
         cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldc) * 4};
@@ -1081,7 +1082,7 @@ int host_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
         return ee == cudaSuccess;
     };
 
-    // Large problems are cut into a grid of up to 8 x 8 blocks of C (1024 rows / columns or more each), and three streams work on them at
+    // Large problems are cut into a grid of up to 4 x 4 blocks of C (1024 rows / columns or more each), and three streams work on them at
     // once: one copies row blocks of A and column blocks of B in (in the order the blocks of C need them),
     // the caller's stream computes block after block, one copies finished blocks out -- so both directions
     // of the host link are busy while the kernels run, and the first block starts after two operand
@@ -1092,8 +1093,12 @@ int host_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     if (K > 0 && total_bytes >= (32LL << 20) && dev->copy_in && dev->copy_out) {
         bi = static_cast<int>(M / 1024 < 1 ? 1 : (M / 1024 > kHostBlocks ? kHostBlocks : M / 1024));
         bj = static_cast<int>(N / 1024 < 1 ? 1 : (N / 1024 > kHostBlocks ? kHostBlocks : N / 1024));
-        static const int max_bi = env_int("MIPGEMM_HOST_ROW_BLOCKS", kHostBlocks);
-        static const int max_bj = env_int("MIPGEMM_HOST_COL_BLOCKS", kHostBlocks);
+        // (measured on the square sweep: 4 x 4 blocks beat 8 x 4, 8 x 2, 4 x 2, 2 x 4 and row blocks only --
+        // narrower blocks make the pitched copies of C slower, fewer blocks lengthen the head)
+        static const int max_bi = env_int("MIPGEMM_HOST_ROW_BLOCKS", 4);
+        static const int max_bj = env_int("MIPGEMM_HOST_COL_BLOCKS", 4);
+        if (bi > kHostBlocks) bi = kHostBlocks;
+        if (bj > kHostBlocks) bj = kHostBlocks;
         if (bi > max_bi) bi = max_bi < 1 ? 1 : max_bi;
         if (bj > max_bj) bj = max_bj < 1 ? 1 : max_bj;
     }
@@ -1281,11 +1286,42 @@ int mipgemm_conv_u8s8s32(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t 
         cudaError_t e = launch_weight_slots(Wt, wp, Cout, R, seg, slot, stream);
         ++g_launches;
         if (e != cudaSuccess) return cuda_fail(e);
-        const Plan pl = make_plan(M, Cout, Kp, block_k, dev, 64, 64, /*one_cta_no_split=*/true);
+        Plan pl = make_plan(M, Cout, Kp, block_k, dev, 64, 64, /*one_cta_no_split=*/true);
+        // Staged form: image rows that are multiples of 16 bytes (bulk copies) and few enough per tile go through
+        // two row buffers in shared memory, which the pipeline stages make room for.
+        const long long row_bytes = g.W * g.Cin;
+        const int span = (R - 1) * dil_h + 1;
+        const int rows_max = static_cast<int>((kBlockM - 2) / g.Wo + 2);
+        const long long payload = static_cast<long long>(rows_max) * span * row_bytes;
+        const long long rowbuf_stride = round_up(payload + slot + 64, 128);
+        const int stage_bytes_g = kBlockM * block_k + pl.block_n * block_k;
+        const long long table_bytes = 8LL * 8 * ((Kp + block_k - 1) / block_k);      // one entry per 16-byte chunk of A
+        const long long room = kSmemBudget - kCtrlBytes - kStagingBytes - 1024 - (64 + 2 * rowbuf_stride + table_bytes);
+        const bool staged = MIP_ENV_KNOB("MIPGEMM_NO_STAGED_GATHER", 0) == 0 && row_bytes % 16 == 0 &&
+                            reinterpret_cast<uintptr_t>(X) % 16 == 0 && pad_w * g.Cin + 4 <= 64 && payload <= 48 * 1024 &&
+                            span <= 4095 && slot <= 8192 &&
+                            room >= 3LL * stage_bytes_g;
+        if (staged && pl.stages > room / stage_bytes_g) pl.stages = static_cast<int>(room / stage_bytes_g);
         DenseParams p;
         std::memset(&p, 0, sizeof(p));
         fill_common(p, pl, M, Cout, Y, Cout, block_k, true, accumulate, dev);
         p.a_gather = 1;
+        p.g_staged = staged ? 1 : 0;
+        p.g_span = span;
+        p.g_rows_max = rows_max;
+        p.g_rowbuf_stride = static_cast<int>(rowbuf_stride);
+        p.g_r = R;
+        p.g_ho = static_cast<int>(g.Ho);
+        p.g_table_bytes = static_cast<int>(table_bytes);
+        auto magic = [](long long d, uint32_t* mul, uint32_t* shift) {      // q = (umulhi(mul, n) + n) >> shift, n < 2^31
+            uint32_t l = 0;
+            while ((1LL << l) < d) ++l;
+            *mul = static_cast<uint32_t>(((1ULL << 32) * ((1ULL << l) - static_cast<unsigned long long>(d))) /
+                                         static_cast<unsigned long long>(d) + 1);
+            *shift = l;
+        };
+        magic(g.Wo, &p.g_wo_mul, &p.g_wo_shift);
+        magic(g.Ho, &p.g_ho_mul, &p.g_ho_shift);
         p.gx = X;
         p.g_xbytes = g.Nb * g.H * g.W * g.Cin;
         p.g_h = static_cast<int>(g.H);

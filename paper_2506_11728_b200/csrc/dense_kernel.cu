@@ -384,6 +384,10 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
     const uint32_t bar_tfull = bar_empty + 8u * p.stages;
     const uint32_t bar_tempty = bar_tfull + 16u;
     const uint32_t bar_drain = bar_tempty + 16u;
+    // staged gather: two more barrier pairs at ctrl + 256, the two image-row buffers behind the control block
+    const uint32_t bar_rows_full = ctrl + 256u;
+    const uint32_t bar_rows_empty = ctrl + 272u;
+    const uint32_t rowbuf0 = ctrl + kCtrlBytes + 64u;      // (64 guard bytes in front: windows start left of a row)
     uint8_t* ctrl_ptr = smem + p.stages * stage_bytes + kStagingBytes;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctrl_ptr + 16 * p.stages + 40);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(tmem_slot + 1);
@@ -404,6 +408,12 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             mbar_init(bar_tempty + 8u * a, kPair ? 2 * kEpiWarps : kEpiWarps);
         }
         mbar_init(bar_drain, 1);
+        if (kGather) {
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(bar_rows_full + 8u * b, 1);
+                mbar_init(bar_rows_empty + 8u * b, 4 * kGatherParities);   // one arrival per gather warp
+            }
+        }
         *abort_flag = 0;
         fence_mbar_init();
         if (!kGather) tma_prefetch_desc(&p.tmap_a);
@@ -432,6 +442,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
     const int total_units = p.tiles_m * p.tiles_n * p.split_k * (p.batch > 1 ? p.batch : 1);
     const uint64_t budget = p.wait_budget_ns;
     uint32_t issued = 0;   // producer warp: k-blocks whose loads have been issued (the unwinding path needs it)
+    uint32_t rows_tiles = 0;   // producer warp, staged gather: tiles whose image rows have been requested
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (whole warp loops)
@@ -453,6 +464,34 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 const int wo = rem - ho * p.conv_wo;
                 cw = wo * p.stride_w - p.pad_w;
                 chh = ho * p.stride_h - p.pad_h;
+            }
+            if (kGather && p.g_staged) {
+                // Staged gather: request the image rows this tile's output pixels read.  Output row L (counted
+                // through the whole batch) owns g_span row slots of the buffer; slot r * dil_h of them holds input
+                // row ho * stride_h - pad_h + r * dil_h if that row exists.
+                const uint32_t buf = rows_tiles & 1u, rph = (rows_tiles >> 1) & 1u;
+                if (!mbar_wait(bar_rows_empty + 8u * buf, rph ^ 1u, abort_flag, budget)) { ok = false; break; }
+                if (elect_one()) {
+                    const uint32_t rows_full = bar_rows_full + 8u * buf;
+                    const uint32_t dst0 = rowbuf0 + buf * static_cast<uint32_t>(p.g_rowbuf_stride);
+                    const int L0 = tc.m0 / p.conv_wo;
+                    const int L1 = (min(tc.m0 + kBlockM, p.M) - 1) / p.conv_wo;
+                    for (int L = L0; L <= L1; ++L) {
+                        const int n_img = L / p.g_ho;
+                        const int hb = (L - n_img * p.g_ho) * p.stride_h - p.pad_h;
+                        for (int r = 0; r < p.g_r; ++r) {
+                            const int h = hb + r * p.dil_h;
+                            if (h >= 0 && h < p.g_h) {
+                                mbar_expect_tx(rows_full, static_cast<uint32_t>(p.g_row_bytes));
+                                bulk_load_1d(dst0 + static_cast<uint32_t>(((L - L0) * p.g_span + r * p.dil_h) * p.g_row_bytes),
+                                             p.gx + static_cast<long long>(n_img * p.g_h + h) * p.g_row_bytes,
+                                             static_cast<uint32_t>(p.g_row_bytes), rows_full);
+                            }
+                        }
+                    }
+                    mbar_arrive(rows_full);
+                }
+                ++rows_tiles;
             }
             int tap = 0, cc = 0, fr = 0, fs = 0;
             if (p.a_im2col) {
@@ -580,6 +619,100 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         const int row = ((warp - kGatherFirstWarp) & 3) * 32 + lane;
         const int parity = (warp - kGatherFirstWarp) >> 2;
         constexpr int kCh = 8 / kGatherParities;        // chunks per thread and k-block
+        if (p.g_staged) {
+            // Staged form: the rows this tile reads are in shared memory (see the producer warp); a chunk is five
+            // aligned 4-byte shared-memory loads, four funnel shifts and one swizzled 16-byte store.  The warps
+            // are bound by their instruction count, so everything that does not depend on the pixel is looked
+            // up: a table in shared memory holds, for every 16-byte chunk q of a row of A, its byte offset from
+            // the window's first byte (filter row * image row pitch + offset in the slot), the filter row's
+            // distance in image rows and the offset in the slot; the two divisions per pixel use multipliers
+            // prepared by the host.
+            constexpr int kStrideB = 16 * kGatherParities;
+            const bool fixed = kStrideB % p.g_slot == 0;     // every chunk of this thread at the same offset in its slot
+            const uint32_t tab = rowbuf0 + 2u * static_cast<uint32_t>(p.g_rowbuf_stride);
+            {
+                const int entries = p.k_blocks * 8;
+                for (int q = static_cast<int>(threadIdx.x) - 32 * kGatherFirstWarp; q < entries; q += 128 * kGatherParities) {
+                    const int r = (q * 16) / p.g_slot;
+                    const int off = q * 16 - r * p.g_slot;
+                    const bool valid = q < p.g_chunks && off < p.g_seg;
+                    // (chunks of the padding behind the last slot read the window's first bytes and are cleared)
+                    const uint32_t lo32 = valid ? static_cast<uint32_t>(r * p.dil_h * p.g_row_bytes + off) : 0u;
+                    const uint32_t hi32 = valid ? (static_cast<uint32_t>(r * p.dil_h) | (static_cast<uint32_t>(off) << 12))
+                                                : 0x80000000u;
+                    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(tab + 8u * q), "r"(lo32), "r"(hi32) : "memory");
+                }
+                asm volatile("bar.sync 2, %0;" ::"n"(128 * kGatherParities) : "memory");     // the gather warps only
+            }
+            const int off_c = (parity * 16) % p.g_slot;      // (fixed case) this thread's offset in its slots
+            uint32_t s = 0, phase = 0, tile_no = 0;
+            bool ok = true;
+            for (int unit = first_unit; unit < total_units && ok; unit += unit_stride, ++tile_no) {
+                const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
+                const int m = tc.m0 + row;
+                const uint32_t mm = static_cast<uint32_t>(m < p.M ? m : tc.m0);
+                const uint32_t L = (__umulhi(p.g_wo_mul, mm) + mm) >> p.g_wo_shift;     // output row, counted through the batch
+                const uint32_t L0 = (__umulhi(p.g_wo_mul, static_cast<uint32_t>(tc.m0)) + static_cast<uint32_t>(tc.m0)) >> p.g_wo_shift;
+                const int wo = static_cast<int>(mm - L * static_cast<uint32_t>(p.conv_wo));
+                const uint32_t n_img = (__umulhi(p.g_ho_mul, L) + L) >> p.g_ho_shift;
+                const int h0 = static_cast<int>(L - n_img * static_cast<uint32_t>(p.g_ho)) * p.stride_h - p.pad_h;
+                const int wb = (wo * p.stride_w - p.pad_w) * p.g_cin;     // window start, bytes into the image row
+                const int lo = max(0, -wb);
+                const int hi = (p.g_row_bytes - wb >= p.g_seg) ? p.g_slot : p.g_row_bytes - wb;
+                const uint32_t buf = tile_no & 1u;
+                // address of byte 0 of slot 0 of this pixel's window (may lie a few bytes left of its row)
+                const int base = static_cast<int>(rowbuf0) + static_cast<int>(buf) * p.g_rowbuf_stride +
+                                 static_cast<int>(L - L0) * p.g_span * p.g_row_bytes + wb;
+                uint4 tile_mask = make_uint4(~0u, ~0u, ~0u, ~0u);
+                bool row_ok = m < p.M;
+                if (fixed) {
+                    tile_mask = gather_mask(lo - off_c, hi - off_c);
+                    row_ok = row_ok & (off_c < hi) & (off_c + 16 > lo);
+                }
+                if (!mbar_wait(bar_rows_full + 8u * buf, (tile_no >> 1) & 1u, abort_flag, budget)) { ok = false; break; }
+                for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb) {
+                    if (!mbar_wait(bar_empty + 8u * s, phase ^ 1u, abort_flag, budget)) { ok = false; break; }
+                    const uint32_t dst = smem_base + s * stage_bytes + static_cast<uint32_t>(row) * 128u;
+#pragma unroll
+                    for (int c = 0; c < kCh; ++c) {
+                        const int j = parity + kGatherParities * c;            // chunk within the k-block
+                        uint32_t e_lo, e_hi;
+                        asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(e_lo), "=r"(e_hi)
+                                     : "r"(tab + 8u * static_cast<uint32_t>(kb * 8 + j)) : "memory");
+                        const int h = h0 + static_cast<int>(e_hi & 0xFFFu);
+                        bool use = row_ok & (static_cast<int>(e_hi) >= 0) &
+                                   (static_cast<unsigned>(h) < static_cast<unsigned>(p.g_h));
+                        uint4 mk = tile_mask;
+                        if (!fixed) {
+                            const int off = static_cast<int>((e_hi >> 12) & 0x3FFFu);
+                            use = use & (off < hi) & (off + 16 > lo);
+                            mk = gather_mask(lo - off, hi - off);
+                        }
+                        const uint32_t a = static_cast<uint32_t>(base + static_cast<int>(e_lo));
+                        const uint32_t al = a & ~3u;
+                        const uint32_t sh = (a & 3u) * 8u;
+                        uint32_t x[5];
+#pragma unroll
+                        for (int i = 0; i < 5; ++i)
+                            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(x[i]) : "r"(al + 4u * i) : "memory");
+                        const uint32_t keep = use ? ~0u : 0u;
+                        uint32_t vv[4];
+                        vv[0] = __funnelshift_r(x[0], x[1], sh) & (mk.x & keep);
+                        vv[1] = __funnelshift_r(x[1], x[2], sh) & (mk.y & keep);
+                        vv[2] = __funnelshift_r(x[2], x[3], sh) & (mk.z & keep);
+                        vv[3] = __funnelshift_r(x[3], x[4], sh) & (mk.w & keep);
+                        st_shared_v4(dst + (static_cast<uint32_t>(j ^ (row & 7)) << 4), vv);
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_full + 8u * s);
+                    if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                __syncwarp();                                   // every lane has read its last bytes of the row buffer
+                if (lane == 0) mbar_arrive(bar_rows_empty + 8u * buf);
+            }
+        } else {
         const int xbytes = static_cast<int>(p.g_xbytes);
         const uint32_t align = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(p.gx)) & 3u;
         constexpr int kNone = -0x40000000;
@@ -697,6 +830,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_full + 8u * s);
             if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
+        }
         }
     } else if (warp < 2 + kEpiWarps) {
         // ------------------------------------------------------------ epilogue
@@ -893,6 +1027,15 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         //    landed (a peer CTA cannot observe its own copies -- they complete on the leader's barrier; it is
         //    held by the cluster barrier below until the leader has finished here);
         //  * the MMA warp lets every MMA it issued retire (one more commit, bounded wait).
+        if (kGather && warp == 0 && p.g_staged) {       // image rows requested for the last two tiles
+            for (uint32_t i = 1; i <= min(rows_tiles, 2u); ++i) {
+                const uint32_t t = rows_tiles - i;
+                const uint64_t t0 = globaltimer_ns();
+                while (!mbar_try_wait(bar_rows_full + 8u * (t & 1u), (t >> 1) & 1u)) {
+                    if (globaltimer_ns() - t0 > budget) break;
+                }
+            }
+        }
         if (warp == 0 && leader) {
             const uint32_t n = min(issued, static_cast<uint32_t>(p.stages));
             for (uint32_t i = 1; i <= n; ++i) {

@@ -96,6 +96,17 @@ struct alignas(64) DenseParams {
     int g_h, g_row_bytes;    // image rows, bytes per image row (W * Cin)
     int g_cin, g_seg, g_slot;
     int g_chunks;            // 16-byte chunks per row of A (R * g_slot / 16)
+    // staged form of the gather (image rows are multiples of 16 bytes and few enough fit shared memory): the
+    // producer warp copies the input rows a tile needs into one of two row buffers with bulk copies, and the
+    // gather warps realign from shared memory instead of from global memory.  Output row o of the tile
+    // (o = 0 .. g_rows_max-1) owns g_span = (R-1)*dil_h + 1 consecutive slots of g_row_bytes.
+    int g_staged;
+    int g_span, g_rows_max;
+    int g_rowbuf_stride;     // bytes between the two row buffers (payload + guard bytes, multiple of 128)
+    int g_table_bytes;       // chunk table behind the row buffers: 8 bytes per 16-byte chunk of a (padded) row of A
+    int g_r, g_ho;           // filter rows, output rows per image
+    // exact division of any n < 2^31 by Wo and by Ho without a divide: q = (umulhi(mul, n) + n) >> shift
+    uint32_t g_wo_mul, g_wo_shift, g_ho_mul, g_ho_shift;
     unsigned int* status;    // device word, bit 0 set when a bounded wait expired
     unsigned long long wait_budget_ns;
     int debug_flags;         // test hook (mipgemm_debug_set): bit 0 = never signal "accumulator ready"

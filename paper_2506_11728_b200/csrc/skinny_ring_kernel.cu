@@ -299,9 +299,12 @@ cudaError_t launch_ring_t(SkinnyRingParams p, int grid, cudaStream_t stream) {
         const int fit_min = MIP_ENV_KNOB("MIPGEMM_RING_FIT_MIN", 2);
         const int const_grid = MIP_ENV_KNOB("MIPGEMM_RING_CONST_GRID", 0);
         const int budget = 228 * 1024 / 2 - 2048;
-        const int fit = (budget - fixed - tok_bytes) / kSlotBytes;
+        // (experiment: tokens of calls with M <= this many rows are read from global memory, chunk by chunk)
+        const int tok_global = MIP_ENV_KNOB("MIPGEMM_RING_TOKENS_GLOBAL", 0);
+        const bool from_global = p.M <= tok_global;
+        const int fit = (budget - fixed - (from_global ? 0 : tok_bytes)) / kSlotBytes;
         if (fit >= fit_min) {
-            p.tokens_in_smem = 1;
+            p.tokens_in_smem = from_global ? 0 : 1;
             slots = fit < kMaxRingSlots ? fit : kMaxRingSlots;
             const int units = (p.N + 15) / 16;
             const int cap = (const_grid && p.b_constant) ? grid : 2 * grid;

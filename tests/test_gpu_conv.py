@@ -78,6 +78,12 @@ GATHER_CASES = [
     (2, 11, 10, 7, 33, 4, 3, (3, 2), (0, 2), (1, 1)),        # padding only in w, stride 3
     (1, 40, 40, 100, 48, 3, 3, (1, 1), (1, 1), (1, 1)),      # long rows of A: K' = 912, 8 k-blocks
     (1, 5, 5, 3, 4, 3, 3, (1, 1), (1, 1), (1, 1)),           # the whole batch is 75 bytes
+    # image rows that are multiples of 16 bytes: staged in shared memory by bulk copies
+    (3, 20, 16, 3, 64, 7, 7, (2, 2), (3, 3), (1, 1)),        # 48-byte rows; tiles straddle output rows and images
+    (2, 16, 32, 4, 32, 5, 5, (1, 2), (2, 2), (1, 1)),        # 128-byte rows, slot 32, stride only in w
+    (1, 12, 16, 5, 7, 3, 2, (2, 1), (1, 0), (2, 1)),         # 80-byte rows, dilated filter rows, Cout % 4 != 0
+    (2, 8, 8, 2, 16, 8, 8, (1, 1), (4, 4), (1, 1)),          # filter as large as the image, padding on all sides
+    (5, 4, 16, 1, 8, 3, 3, (1, 1), (1, 1), (1, 1)),          # tiny images: a tile spans several of them
 ]
 
 

@@ -171,3 +171,35 @@ def test_two_host_threads_on_two_streams(mg):
             want = orc.gemm(A, B, M, N, K)
             got = dC.cpu().numpy()
             assert np.array_equal(got, want), (mode, M, N, K, first_mismatch(got.reshape(M, N), want.reshape(M, N)))
+
+
+def test_dispatch_log_names_the_path_taken():
+    """MIPGEMM_LOG=1 prints one line per call with the dispatch decision (read at library load, hence a child
+    process)."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = (
+        "import torch\n"
+        "from paper_2506_11728_b200 import binding as mg\n"
+        "a = torch.zeros(1 << 22, dtype=torch.int8, device='cuda')\n"
+        "c = torch.empty(1 << 22, dtype=torch.int32, device='cuda')\n"
+        "mg.mipgemm_s8s8s32(512, 512, 512, a, 512, a, 512, c, 512, 0)\n"
+        "mg.mipgemm_s8s8s32(512, 512, 512, a, 512, a, 512, c, 512, 0)\n"
+        "mg.mipgemm_s8s8s32(4, 4096, 1024, a, 1024, a, 1024, c, 4096, 0)\n"
+        "mg.mipgemm_u8s8s32(100, 200, 77, a, 77, a, 77, c, 200, 1)\n"
+        "mg.mipgemm_conv_u8s8s32(2, 14, 14, 128, 64, 3, 3, 1, 1, 1, 1, 1, 1, a, a, c, 0)\n"
+        "mg.mipgemm_conv_u8s8s32(2, 32, 32, 3, 64, 7, 7, 2, 2, 3, 3, 1, 1, a, a, c, 0)\n"
+        "assert mg.mipgemm_device_status() == mg.OK\n")
+    env = dict(os.environ, MIPGEMM_LOG="1", PYTHONPATH=root)
+    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stderr.splitlines() if l.startswith("mipgemm:")]
+    assert len(lines) == 6, lines
+    assert "gemm s8 M=512 N=512 K=512 -> dense" in lines[0] and "plan=new" in lines[0]
+    assert "plan=cached" in lines[1]
+    assert "skinny" in lines[2]
+    assert "re-pitched" in lines[3] and "accumulate" in lines[3]
+    assert "conv (TMA im2col)" in lines[4]
+    assert "conv (gathered im2col)" in lines[5]
