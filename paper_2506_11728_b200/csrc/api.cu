@@ -443,10 +443,8 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
     p.cluster_split = pl.cluster_split;
     const int group_env = MIP_ENV_KNOB("MIPGEMM_GROUP_N", 0);
     const int raster_env = MIP_ENV_KNOB("MIPGEMM_RASTER", 0);
-    const int evict_env = MIP_ENV_KNOB("MIPGEMM_C_EVICT_FIRST", 0);
     p.group_n = group_env > 0 ? group_env : 8;
     p.raster = raster_env;
-    p.c_evict_first = evict_env;
     p.use_red = (pl.split_k > 1 && !pl.cluster_split) ? 1 : 0;
     p.accumulate = p.use_red ? 0 : (accumulate ? 1 : 0);
     const uintptr_t c_addr = reinterpret_cast<uintptr_t>(C);

@@ -197,7 +197,6 @@ __device__ __forceinline__ void tma_store_slab(const DenseParams& p, uint32_t bu
 #endif
     if (issuer && elect_one()) {
         if (p.batch > 1) tma_store_3d(&p.tmap_c, buf, x, y, z);
-        else if (p.c_evict_first) tma_store_2d_hint(&p.tmap_c, buf, x, y, l2_policy_evict_first());
         else tma_store_2d(&p.tmap_c, buf, x, y);
         tma_store_commit();
     }
@@ -400,7 +399,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(bar_full + 8u * s, kGather ? 1 + 4 * kGatherParities : 1);   // + one arrival per gather warp
+            mbar_init(bar_full + 8u * s, kGather ? 1 + 4 * kGatherParities : ((kQ8 && !kGather) ? 1 : 2));   // producer(s) (+ gather warps)
             mbar_init(bar_empty + 8u * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -444,11 +443,21 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
     uint32_t issued = 0;   // producer warp: k-blocks whose loads have been issued (the unwinding path needs it)
     uint32_t rows_tiles = 0;   // producer warp, staged gather: tiles whose image rows have been requested
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer (whole warp loops)
+    // Two producer warps, one per operand (warp 0: A, warp 2 + kEpiWarps: B): a TMA load costs its issuing
+    // thread some 250 clocks, so with both loads of a k-block in one thread the producer itself paced the
+    // shapes with short k-blocks (64-channel convolutions: 2 x 250 clocks against 190 clocks of smem fill).
+    // Both walk the same tiles and stages; each arms the stage's "full" barrier with its own byte count.
+    // (The gather form has one producer: operand A is written by the gather warps.  So has the 8-bit-code form,
+    // whose eight epilogue warps need the registers.)
+    constexpr bool kTwoProducers = !kGather && !kQ8;
+    constexpr int kWarpB = kTwoProducers ? 2 + kEpiWarps : 0;
+    if (warp == 0 || warp == kWarpB) {
+        // ------------------------------------------------------------ TMA producers (whole warp loops)
         uint32_t s = 0, phase = 0;
         bool ok = true;
-        const uint32_t tx_bytes = kGather ? b_bytes : (kPair ? 2u * stage_bytes : stage_bytes);
+        const bool side_a = !kGather && warp == 0;
+        const bool side_b = warp == kWarpB;
+        const uint32_t tx_bytes = (kPair ? 2u : 1u) * ((side_a ? a_bytes : 0u) + (side_b ? b_bytes : 0u));
         for (int unit = first_unit; unit < total_units && ok; unit += unit_stride) {
             const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
             const int m_cta = tc.m0 + static_cast<int>(cta_rank) * kBlockM;
@@ -471,25 +480,32 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 // row ho * stride_h - pad_h + r * dil_h if that row exists.
                 const uint32_t buf = rows_tiles & 1u, rph = (rows_tiles >> 1) & 1u;
                 if (!mbar_wait(bar_rows_empty + 8u * buf, rph ^ 1u, abort_flag, budget)) { ok = false; break; }
-                if (elect_one()) {
+                {
+                    // one (output row, filter row) pair per lane: a single thread walking all of them paced the
+                    // whole tile
                     const uint32_t rows_full = bar_rows_full + 8u * buf;
                     const uint32_t dst0 = rowbuf0 + buf * static_cast<uint32_t>(p.g_rowbuf_stride);
-                    const int L0 = tc.m0 / p.conv_wo;
-                    const int L1 = (min(tc.m0 + kBlockM, p.M) - 1) / p.conv_wo;
-                    for (int L = L0; L <= L1; ++L) {
-                        const int n_img = L / p.g_ho;
-                        const int hb = (L - n_img * p.g_ho) * p.stride_h - p.pad_h;
-                        for (int r = 0; r < p.g_r; ++r) {
-                            const int h = hb + r * p.dil_h;
-                            if (h >= 0 && h < p.g_h) {
-                                mbar_expect_tx(rows_full, static_cast<uint32_t>(p.g_row_bytes));
-                                bulk_load_1d(dst0 + static_cast<uint32_t>(((L - L0) * p.g_span + r * p.dil_h) * p.g_row_bytes),
-                                             p.gx + static_cast<long long>(n_img * p.g_h + h) * p.g_row_bytes,
-                                             static_cast<uint32_t>(p.g_row_bytes), rows_full);
-                            }
+                    const uint32_t m0u = static_cast<uint32_t>(tc.m0);
+                    const uint32_t m1u = static_cast<uint32_t>(min(tc.m0 + kBlockM, p.M) - 1);
+                    const uint32_t L0 = (__umulhi(p.g_wo_mul, m0u) + m0u) >> p.g_wo_shift;
+                    const uint32_t L1 = (__umulhi(p.g_wo_mul, m1u) + m1u) >> p.g_wo_shift;
+                    const int pairs = static_cast<int>(L1 - L0 + 1) * p.g_r;
+                    for (int idx = lane; idx < pairs; idx += 32) {
+                        const int o = idx / p.g_r;
+                        const int r = idx - o * p.g_r;
+                        const uint32_t L = L0 + static_cast<uint32_t>(o);
+                        const uint32_t n_img = (__umulhi(p.g_ho_mul, L) + L) >> p.g_ho_shift;
+                        const int h = static_cast<int>(L - n_img * static_cast<uint32_t>(p.g_ho)) * p.stride_h - p.pad_h +
+                                      r * p.dil_h;
+                        if (h >= 0 && h < p.g_h) {
+                            mbar_expect_tx(rows_full, static_cast<uint32_t>(p.g_row_bytes));
+                            bulk_load_1d(dst0 + static_cast<uint32_t>((o * p.g_span + r * p.dil_h) * p.g_row_bytes),
+                                         p.gx + (static_cast<long long>(n_img) * p.g_h + h) * p.g_row_bytes,
+                                         static_cast<uint32_t>(p.g_row_bytes), rows_full);
                         }
                     }
-                    mbar_arrive(rows_full);
+                    __syncwarp();                      // every lane's transaction count is in before the arrival
+                    if (lane == 0) mbar_arrive(rows_full);
                 }
                 ++rows_tiles;
             }
@@ -508,8 +524,8 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 const uint32_t a_dst = smem_base + s * stage_bytes;
                 if (elect_one()) {
                     if (leader) mbar_arrive_expect_tx(full_local, tx_bytes);
-                    if (kGather) {
-                        // operand A is written by the gather warps
+                    if (!side_a) {
+                        // operand A is the other producer warp's (or, in the gather form, the gather warps')
                     } else if (p.a_im2col) {
                         if (kPair)
                             tma_load_im2col_4d_pair(a_dst, &p.tmap_a, full, cc * p.block_k, cw, chh, cn,
@@ -529,7 +545,9 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     } else {
                         tma_load_2d(a_dst, &p.tmap_a, full, kb * p.block_k, m_cta);
                     }
-                    if (kMN && p.b_mn) {          // tensor {N, K}: one [k][128 B] block per 128 columns
+                    if (!side_b) {
+                        // operand B is the other producer warp's
+                    } else if (kMN && p.b_mn) {   // tensor {N, K}: one [k][128 B] block per 128 columns
                         for (int blk = 0; blk * 128 < b_rows; ++blk) {
                             const uint32_t dst = a_dst + a_bytes + blk * p.block_k * 128;
                             if (kPair) tma_load_2d_pair(dst, &p.tmap_b, full, n_cta + blk * 128, kb * p.block_k);
@@ -966,7 +984,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         cluster_arrive();
         cluster_wait();
         tc_fence_after();
-        if (warp >= 2 && *abort_flag == 0) {
+        if (warp >= 2 && warp < 2 + kEpiWarps && *abort_flag == 0) {
             for (uint32_t d = 0; d < S; ++d) {
                 if (d == rank) continue;
                 const uint32_t slot = rank < d ? rank : rank - 1;            // my slot among d's S-1 senders
@@ -986,7 +1004,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         }
         cluster_arrive();
         cluster_wait();
-        if (warp >= 2 && *abort_flag == 0) {
+        if (warp >= 2 && warp < 2 + kEpiWarps && *abort_flag == 0) {
             const int m_cta = tc.m0;
             const int row = m_cta + r_tile;
             const uint32_t my_staging = staging + static_cast<uint32_t>(q) * 8192u;

@@ -32,8 +32,8 @@ inline bool live_env() {
                    return ::mip::live_env() ? ::mip::env_int(name, fallback) : cached; }())
 
 constexpr int kBlockM = 128;          // rows of C per CTA (TMEM lanes)
-constexpr int kDenseThreads = 192;    // producer warp, MMA warp, 4 epilogue warps
-constexpr int kDenseQ8Threads = 320;  // 8-bit-code epilogue: 8 epilogue warps
+constexpr int kDenseThreads = 224;    // producer warp (A), MMA warp, 4 epilogue warps, producer warp (B)
+constexpr int kDenseQ8Threads = 320;  // 8-bit-code epilogue: one producer warp, MMA warp, 8 epilogue warps
 // Gather form of the dense kernel: 4 * kGatherParities more warps build operand A from an image;
 // warp w of them takes rows 32*(w%4).. of the tile and every kGatherParities-th 16-byte chunk.
 constexpr int kGatherParities = 4;
@@ -68,7 +68,6 @@ struct alignas(64) DenseParams {
     int cluster_split;       // > 1: the split_k CTAs sharing a tile form a cluster and reduce through DSMEM
     int group_n;             // n-tiles per rasterisation group
     int raster;              // bit 0: serpentine (odd groups are swept bottom to top)
-    int c_evict_first;       // 1: TMA tile stores of C carry an evict-first L2 hint
     int accumulate;          // epilogue adds the incoming C
     int use_red;             // epilogue reduces with red.global.add (split-K)
     int store_vec;           // 8, 4 or 1 int32 per store instruction

@@ -296,19 +296,20 @@ cudaError_t launch_ring_t(SkinnyRingParams p, int grid, cudaStream_t stream) {
         // promise, while the previous call drains) the other keeps streaming, and it no longer matters
         // which call's CTAs the block scheduler puts side by side.  Measured over a chain of 264 decode
         // GEMMs: 2.49 -> 2.28 ms without the promise, 2.06 -> 1.96 ms with it.
-        const int fit_min = MIP_ENV_KNOB("MIPGEMM_RING_FIT_MIN", 2);
-        const int const_grid = MIP_ENV_KNOB("MIPGEMM_RING_CONST_GRID", 0);
+        // Measured and not kept (same-process A/B over the 264-launch decode step): one CTA per SM with nine
+        // slots whenever fewer than three fit beside the tokens (M = 16: 6-8 % slower per launch -- eight
+        // consumer warps per SM are too few); under the promise, at most one half-memory CTA per SM and
+        // call, so that two calls are always co-resident (+18 % on the step: the chain of dependent launches,
+        // not the weight stream, paces the small matrices); tokens of M <= 1/4/8 read from global memory chunk
+        // by chunk instead of copied to shared memory (0 / +2 / +6 %).
+        const int fit_min = 2;
         const int budget = 228 * 1024 / 2 - 2048;
-        // (experiment: tokens of calls with M <= this many rows are read from global memory, chunk by chunk)
-        const int tok_global = MIP_ENV_KNOB("MIPGEMM_RING_TOKENS_GLOBAL", 0);
-        const bool from_global = p.M <= tok_global;
-        const int fit = (budget - fixed - (from_global ? 0 : tok_bytes)) / kSlotBytes;
+        const int fit = (budget - fixed - tok_bytes) / kSlotBytes;
         if (fit >= fit_min) {
-            p.tokens_in_smem = from_global ? 0 : 1;
+            p.tokens_in_smem = 1;
             slots = fit < kMaxRingSlots ? fit : kMaxRingSlots;
             const int units = (p.N + 15) / 16;
-            const int cap = (const_grid && p.b_constant) ? grid : 2 * grid;
-            grid = units < cap ? units : cap;
+            grid = units < 2 * grid ? units : 2 * grid;
         }
     }
     p.slots = slots;
