@@ -183,6 +183,7 @@ int get_device(DeviceState** out) {
             }
             if ((e = dense_init()) != cudaSuccess) return cuda_fail(e);
             if ((e = skinny_ring_init()) != cudaSuccess) return cuda_fail(e);
+            if ((e = skinny_ring16_init()) != cudaSuccess) return cuda_fail(e);
             d.pair_clusters = dense_pair_max_clusters(kSmemBudget);
             if (const char* ds = std::getenv("MIPGEMM_DIRECT_STORE")) g_tuning_no_tma_store = std::atoi(ds) != 0;
             if (const char* cs = std::getenv("MIPGEMM_NO_CLUSTER_SPLIT")) g_tuning_no_cluster_split = std::atoi(cs) != 0;
@@ -646,7 +647,8 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
         tun.force_path != MIPGEMM_PATH_DENSE_PAIR) {
         SkinnyParams sp{A, lda, B, ldb, C, ldc, static_cast<int>(M), static_cast<int>(N),
                         static_cast<int>(K), a_unsigned ? 1 : 0, accumulate ? 1 : 0, tl_out_f32, tl_out_scale};
-        if (skinny_ring_supported(sp, dev->sm_count) && !g_tuning_no_skinny_ring) {
+        const bool ring16 = skinny_ring16_supported(sp, dev->sm_count) && MIP_ENV_KNOB("MIPGEMM_NO_RING16", 0) == 0;
+        if ((ring16 || skinny_ring_supported(sp, dev->sm_count)) && !g_tuning_no_skinny_ring) {
             SkinnyRingParams rp;
             std::memset(&rp, 0, sizeof(rp));
             // the weight matrix's tensor map is remembered like a dense plan (kind 3: only tmap_b is used)
@@ -690,8 +692,15 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
                                  inside_constant_range(B, static_cast<size_t>(N - 1) * ldb + K)) ? 1 : 0;
                 rp.status = dev->status_word;
                 rp.wait_budget_ns = g_wait_budget_ns.load(std::memory_order_relaxed);
-                rp.debug_flags = g_debug_flags.load(std::memory_order_relaxed);
-                cudaError_t e = launch_skinny_ring(rp, dev->sm_count, stream);
+                rp.debug_flags = g_debug_flags.load(std::memory_order_relaxed) |
+                                 (MIP_ENV_KNOB("MIPGEMM_RING_ALWAYS_RELEASE", 0) ? 2 : 0);   // (A/B switch)
+                rp.trace = nullptr;
+#ifdef MIPGEMM_TRACE
+                if (const char* tr = std::getenv("MIPGEMM_TRACE_PTR"))
+                    rp.trace = reinterpret_cast<unsigned long long*>(std::strtoull(tr, nullptr, 10));
+#endif
+                cudaError_t e = ring16 ? launch_skinny_ring16(rp, dev->sm_count, stream)
+                                       : launch_skinny_ring(rp, dev->sm_count, stream);
                 ++g_launches;
                 if (e != cudaSuccess) return cuda_fail(e);
                 tl_last_path = MIPGEMM_PATH_SKINNY | path_flags;

@@ -79,12 +79,18 @@ cudaError_t launch_transpose_repack(const void* src, long long src_pitch, void* 
 }
 
 // ---------------------------------------------------------------- zero fill
+// One 64-bit division per element made the scalar form an ALU kernel (2.9 TB/s); rows that are 16-byte
+// addressable are cleared four elements per store.
+template <bool kVec>
 __global__ void mip_fill_zero_kernel(int32_t* C, long long ldc, long long M, long long N) {
-    const long long total = M * N;
+    const long long per_row = kVec ? N / 4 : N;            // stores per row
+    const long long total = M * per_row;
     for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
          i += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const long long r = i / N;
-        C[r * ldc + (i - r * N)] = 0;
+        const long long r = i / per_row;
+        const long long c = i - r * per_row;
+        if (kVec) reinterpret_cast<int4*>(C + r * ldc)[c] = make_int4(0, 0, 0, 0);
+        else C[r * ldc + c] = 0;
     }
 }
 
@@ -120,8 +126,11 @@ cudaError_t launch_weight_slots(const int8_t* src, int8_t* dst, long long rows, 
 cudaError_t launch_fill_zero(int32_t* C, long long ldc, long long M, long long N, cudaStream_t stream) {
     if (M <= 0 || N <= 0) return cudaSuccess;
     const int threads = 256;
-    const long long blocks = min((M * N + threads - 1) / threads, 148LL * 16);
-    mip_fill_zero_kernel<<<static_cast<unsigned>(blocks), threads, 0, stream>>>(C, ldc, M, N);
+    const bool vec = N % 4 == 0 && ldc % 4 == 0 && reinterpret_cast<uintptr_t>(C) % 16 == 0;
+    const long long stores = vec ? M * (N / 4) : M * N;
+    const long long blocks = min((stores + threads - 1) / threads, 148LL * 16);
+    if (vec) mip_fill_zero_kernel<true><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(C, ldc, M, N);
+    else mip_fill_zero_kernel<false><<<static_cast<unsigned>(blocks), threads, 0, stream>>>(C, ldc, M, N);
     return cudaGetLastError();
 }
 

@@ -145,10 +145,15 @@ struct alignas(64) SkinnyRingParams {
     unsigned int* status;
     unsigned long long wait_budget_ns;
     int debug_flags;             // test hook (mipgemm_debug_set): bit 0 = the first CTA never loads its second chunk
+    unsigned long long* trace;   // timeline stamps of the first and last CTA; only read by builds with -DMIPGEMM_TRACE
 };
 bool skinny_ring_supported(const SkinnyParams& p, int sm_count);
 cudaError_t skinny_ring_init();  // once per device
 cudaError_t launch_skinny_ring(const SkinnyRingParams& p, int sm_count, cudaStream_t stream);
+// Ring form for 9 to 16 tokens (chunk-major walk, token chunks streamed through two buffers).
+bool skinny_ring16_supported(const SkinnyParams& p, int sm_count);
+cudaError_t skinny_ring16_init();  // once per device
+cudaError_t launch_skinny_ring16(const SkinnyRingParams& p, int sm_count, cudaStream_t stream);
 
 // Auxiliary kernels.
 cudaError_t launch_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,

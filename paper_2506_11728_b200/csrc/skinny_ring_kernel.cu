@@ -21,6 +21,14 @@ namespace mip {
 
 namespace {
 
+#ifdef MIPGEMM_TRACE
+// stamps of the first CTA in slots 0.., of the last CTA in slots 16..
+#define RING_STAMP(slot) do { if (p.trace && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) && (threadIdx.x & 31) == 0) \
+    p.trace[(blockIdx.x == 0 ? 0 : 16) + (slot)] = globaltimer_ns(); } while (0)
+#else
+#define RING_STAMP(slot) do { } while (0)
+#endif
+
 constexpr int kMaxRingSlots = 12;
 constexpr int kSlotBytes = 16 * 1024;          // 8 slices x 16 rows x 128 B
 constexpr int kRingConsumers = 8;              // consumer warps = k-slices per chunk
@@ -117,6 +125,7 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
 
     const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0);
     const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) RING_STAMP(0);
     if (threadIdx.x == 0) {
         for (int s = 0; s < kRingSlots; ++s) {
             mbar_init(bar_full + 8u * s, 1);
@@ -133,7 +142,9 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
     // promised constant weights: its loads of B then start while the previous kernel drains.
     __syncthreads();
     if (p.pdl_mode == 1) pdl_launch_dependents();
+    if (warp == 0) RING_STAMP(1);
     if (!(p.b_constant && warp == kRingConsumers)) pdl_wait();
+    if (warp == 0) RING_STAMP(2);
 
     const int units = (p.N + 15) >> 4;
     const int chunks = (p.K + 1023) >> 10;
@@ -149,6 +160,7 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
                 // (test hook, bit 0: CTA 0 leaves out the second chunk of its first unit, so its consumers' wait
                 // for that slot runs out)
                 const bool withheld = (p.debug_flags & 1) && blockIdx.x == 0 && u == 0 && ch == 1;
+                if (u == static_cast<int>(blockIdx.x) && ch == 0) RING_STAMP(3);
                 if (elect_one() && !withheld) {
                     mbar_arrive_expect_tx(bar_full + 8u * s, kSlotBytes);
                     tma_load_3d(ring + s * kSlotBytes, &p.tmap_b, bar_full + 8u * s, 0, u * 16, ch * 8);
@@ -173,6 +185,12 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
 
         uint32_t s = 0, phase = 0;
         bool ok = true;
+        // chunks this CTA streams in all; if they fit the ring, no slot is ever used twice
+        const int my_units = (units - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+        // (only chunks whose slot the producer still needs are released: the proxy fence of a release is
+        // ~150 clocks in the consumers' dependency chain, and the last `slots` chunks of a CTA are its tail)
+        const int my_chunks = my_units * chunks;
+        int chunk_no = 0;
         const uint32_t sx0 = tok_base + g * tok_pitch, sx1 = tok_base + (g + 8) * tok_pitch;
         const bool tsm = p.tokens_in_smem != 0;
         if (tsm) {
@@ -180,10 +198,13 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
             // as one bulk copy per token row, all in flight at once (this sits on the critical
             // path right after the previous kernel's completion, and L2 round trips are long
             // while every SM streams weights).
-            if (threadIdx.x == 0) {
-                mbar_arrive_expect_tx(bar_tokens, static_cast<uint32_t>(p.M) * static_cast<uint32_t>(p.K));
-                for (int r = 0; r < p.M; ++r)
-                    bulk_load_1d(tok_base + r * tok_pitch, A + static_cast<long long>(r) * p.lda,
+            // (one lane per token row: issuing a bulk copy costs its thread a few hundred clocks, and this sits
+            // right behind the previous kernel's completion)
+            if (warp == 0) {
+                if (lane == 0) mbar_arrive_expect_tx(bar_tokens, static_cast<uint32_t>(p.M) * static_cast<uint32_t>(p.K));
+                __syncwarp();
+                if (lane < p.M)
+                    bulk_load_1d(tok_base + lane * tok_pitch, A + static_cast<long long>(lane) * p.lda,
                                  static_cast<uint32_t>(p.K), bar_tokens);
             }
             ok = mbar_wait(bar_tokens, 0u, abort_flag, budget);
@@ -192,20 +213,25 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
         // whether to go on is decided by all 256 together (here and at the end of every unit), so that no warp
         // can leave while another still expects it at a barrier.
         ok = !named_bar_or(1, 256, !ok);
+        if (warp == 0) RING_STAMP(4);
         TokenRegs cur = {}, nxt;
         if (ok) {
             if (tsm) load_tokens_smem<kSecondTokenBlock>(cur, sx0, sx1, warp, p.K, t, tok0_ok, tok1_ok);
             else load_tokens<kSecondTokenBlock>(cur, x0, x1, warp, p.K, t, tok0_ok, tok1_ok);
         }
         for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
-            int acc0[4] = {0, 0, 0, 0};
-            int acc1[4] = {0, 0, 0, 0};
+            // two independent accumulator chains per token block (even / odd k-steps): a chunk's MMAs then
+            // depend on each other two deep instead of four deep
+            int acc0[4] = {0, 0, 0, 0}, acc0b[4] = {0, 0, 0, 0};
+            int acc1[4] = {0, 0, 0, 0}, acc1b[4] = {0, 0, 0, 0};
             for (int ch = 0; ch < chunks; ++ch) {
                 // tokens of the next chunk (the first chunk again after the last) travel while we wait
                 const int next_ch = ch + 1 < chunks ? ch + 1 : 0;
                 if (tsm) load_tokens_smem<kSecondTokenBlock>(nxt, sx0, sx1, next_ch * 8 + warp, p.K, t, tok0_ok, tok1_ok);
                 else load_tokens<kSecondTokenBlock>(nxt, x0, x1, next_ch * 8 + warp, p.K, t, tok0_ok, tok1_ok);
                 if (!mbar_wait(bar_full + 8u * s, phase, abort_flag, budget)) { ok = false; break; }
+                if (warp == 0 && u == static_cast<int>(blockIdx.x) && ch == 0) RING_STAMP(5);
+                if (warp == 0 && u + static_cast<int>(gridDim.x) >= units && ch == chunks - 1) RING_STAMP(6);
                 const uint32_t base = ring + s * kSlotBytes;
                 const uint4 w_ll = lds128(base + off_ll), w_hl = lds128(base + off_hl);
                 const uint4 w_lh = lds128(base + off_lh), w_hh = lds128(base + off_hh);
@@ -214,23 +240,31 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
                 // barrier arrive alone does not wait for loads still queued in the shared-memory
                 // pipe (with two CTAs per SM and weights coming from the L2 the refill did overtake
                 // them), the proxy fence does.
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_empty + 8u * s);      // the slot may be refilled
+                if (chunk_no + kRingSlots < my_chunks || (p.debug_flags & 2)) {   // this slot will be refilled
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_empty + 8u * s);      // the slot may be refilled
+                }
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    ring_mma<kUnsignedTokens>(acc0, word(w_ll, q), word(w_hl, q), word(w_lh, q), word(w_hh, q),
+                    ring_mma<kUnsignedTokens>((q & 1) ? acc0b : acc0, word(w_ll, q), word(w_hl, q), word(w_lh, q), word(w_hh, q),
                                               word(cur.x0l, q), word(cur.x0h, q));
                     if (kSecondTokenBlock)
-                        ring_mma<kUnsignedTokens>(acc1, word(w_ll, q), word(w_hl, q), word(w_lh, q), word(w_hh, q),
+                        ring_mma<kUnsignedTokens>((q & 1) ? acc1b : acc1, word(w_ll, q), word(w_hl, q), word(w_lh, q), word(w_hh, q),
                                                   word(cur.x1l, q), word(cur.x1h, q));
                 }
                 cur = nxt;
+                ++chunk_no;
                 if (++s == static_cast<uint32_t>(kRingSlots)) { s = 0; phase ^= 1u; }
             }
             // (a warp that gave up still brings its partials -- garbage then -- to the barrier below)
             // accumulator fragment: d0 (row g, col 2t), d1 (g, 2t+1), d2 (g+8, 2t), d3 (g+8, 2t+1);
             // row = weight row of the unit, col = token
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                acc0[e] += acc0b[e];
+                acc1[e] += acc1b[e];
+            }
             red[warp][g][2 * t] = acc0[0];
             red[warp][g][2 * t + 1] = acc0[1];
             red[warp][g + 8][2 * t] = acc0[2];
@@ -273,6 +307,7 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
         }
     }
     __syncthreads();
+    if (threadIdx.x == 0) RING_STAMP(7);
     if (threadIdx.x == 0 && *abort_flag != 0) atomicOr(p.status, 1u);
 }
 

@@ -60,11 +60,13 @@ def test_dense_kernel_wait_runs_out_and_the_kernel_returns(mg):
     assert mg.mipgemm_device_status() == mg.OK
 
 
-def test_skinny_ring_wait_runs_out_and_the_kernel_returns(mg):
-    """Skinny ring kernel: its first CTA never loads the second k-chunk of its first unit, so its consumer
-    warps' wait for that slot runs out; all 256 consumer threads decide together to leave."""
+@pytest.mark.parametrize("M", [4, 16])
+def test_skinny_ring_wait_runs_out_and_the_kernel_returns(mg, M):
+    """Skinny ring kernels (the form for up to 8 tokens and the one for 9 to 16): the first CTA never loads the
+    second k-chunk of its first unit, so its consumer warps' wait for that slot runs out; all 256 consumer
+    threads decide together to leave."""
     import torch
-    M, N, K = 4, 4096, 4096
+    N, K = 4096, 4096
     A, B = inputs.uniform_s8(M * K, 71), inputs.uniform_s8(N * K, 72)
     dA, _ka = to_dev(A)
     dB, _kb = to_dev(B)
