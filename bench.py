@@ -724,7 +724,7 @@ def calibrate_fraction(problems, target_s):
     p = problems[min(2, len(problems) - 1)]
     M, N, K = p.dims
     A, B = p.host[0], p.host[1]
-    r = min(M, 8)
+    r = min(M, 128)                                    # (enough rows for every oracle thread to get some)
     orc.gemm(A[:r * K], B, r, N, K)                    # builds / warms the oracle
     t0 = time.perf_counter()
     orc.gemm(A[:r * K], B, r, N, K)
