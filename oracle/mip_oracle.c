@@ -192,6 +192,30 @@ void mip_oracle_requant(const int32_t *Cq, int64_t count, float scale, int32_t l
     }
 }
 
+/*
+ * Per-output-channel integer bias, added to the exact integer sums before they are scaled (the usual
+ * companion of the paper's scale-only scheme, Section 7.3: with the bias quantised at the scale
+ * s_A s_B the real result is C^r = s_A s_B (C^q + b^q); the paper itself carries no bias, so this is
+ * an extension).  out(i,j) = Cq(i,j) + bias[j], computed in int64 and range-checked into int32 like
+ * every other sum here.  Cq and out are rows x cols, dense.  Returns the number of cells whose exact
+ * value does not fit int32 (their low 32 bits are stored), or -1 on invalid arguments.
+ */
+int64_t mip_oracle_add_bias(const int32_t *Cq, int64_t rows, int64_t cols, const int32_t *bias, int32_t *out)
+{
+    if (rows < 0 || cols < 0 || (rows > 0 && cols > 0 && (!Cq || !bias || !out)))
+        return -1;
+    int64_t overflow_cells = 0;
+    for (int64_t i = 0; i < rows; ++i) {
+        for (int64_t j = 0; j < cols; ++j) {
+            int64_t v = (int64_t)Cq[i * cols + j] + (int64_t)bias[j];
+            if (v < (int64_t)INT32_MIN || v > (int64_t)INT32_MAX)
+                overflow_cells += 1;
+            out[i * cols + j] = (int32_t)(uint32_t)(uint64_t)v;
+        }
+    }
+    return overflow_cells;
+}
+
 #ifdef _OPENMP
 #include <omp.h>
 int mip_oracle_threads(void) { return omp_get_max_threads(); }

@@ -68,6 +68,8 @@ def _load():
         lib.mip_oracle_dequant.argtypes = [vp, i64, ctypes.c_double, vp]
         lib.mip_oracle_requant.restype = None
         lib.mip_oracle_requant.argtypes = [vp, i64, ctypes.c_float, ctypes.c_int32, ctypes.c_int32, vp]
+        lib.mip_oracle_add_bias.restype = i64
+        lib.mip_oracle_add_bias.argtypes = [vp, i64, i64, vp, vp]
         lib.mip_oracle_threads.restype = ci
         lib.mip_oracle_threads.argtypes = []
         _lib = lib
@@ -188,4 +190,22 @@ def requant(Cq: np.ndarray, scale: float, lo: int, hi: int) -> np.ndarray:
     flat = np.ascontiguousarray(Cq).reshape(-1)
     out = np.empty(flat.size, dtype=np.int32)
     _load().mip_oracle_requant(_ptr(flat), flat.size, float(np.float32(scale)), int(lo), int(hi), _ptr(out))
+    return out.reshape(Cq.shape)
+
+
+def add_bias(Cq: np.ndarray, bias: np.ndarray, allow_overflow: bool = False) -> np.ndarray:
+    """Cq(..., j) + bias[j], exact (int64, range-checked into int32); the last axis of Cq is the channel axis."""
+    if Cq.dtype != np.int32 or bias.dtype != np.int32:
+        raise TypeError("Cq and bias must be int32")
+    cols = Cq.shape[-1]
+    if bias.shape != (cols,):
+        raise ValueError("bias must have one entry per output channel")
+    flat = np.ascontiguousarray(Cq).reshape(-1, cols)
+    bias = np.ascontiguousarray(bias)
+    out = np.empty_like(flat)
+    rc = _load().mip_oracle_add_bias(_ptr(flat), flat.shape[0], cols, _ptr(bias), _ptr(out))
+    if rc < 0:
+        raise ValueError("mip_oracle_add_bias rejected its arguments")
+    if rc > 0 and not allow_overflow:
+        raise OracleOverflow("%d cells do not fit int32" % rc)
     return out.reshape(Cq.shape)

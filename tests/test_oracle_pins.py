@@ -414,3 +414,35 @@ def test_requant_saturates_and_keeps_shape():
     assert orc.requant(Cq, 1e-9, 0, 255).tolist() == [[2, 0, 1], [0, 0, 0]]
     with pytest.raises(ValueError):
         orc.requant(Cq, float("inf"), -128, 127)
+
+
+# ---------------------------------------------------------------- per-channel bias
+def test_bias_closed_forms_and_numpy():
+    rng = np.random.default_rng(5)
+    Cq = rng.integers(-(1 << 30), 1 << 30, size=(7, 5), dtype=np.int64).astype(np.int32)
+    assert np.array_equal(orc.add_bias(Cq, np.zeros(5, np.int32)), Cq)                     # zero bias: identity
+    bias = rng.integers(-(1 << 20), 1 << 20, size=5, dtype=np.int64).astype(np.int32)
+    assert np.array_equal(orc.add_bias(Cq, bias), (Cq.astype(np.int64) + bias.astype(np.int64)).astype(np.int32))
+    one_hot = np.array([0, 0, 9, 0, 0], np.int32)                                          # only column 2 moves
+    moved = orc.add_bias(Cq, one_hot)
+    assert np.array_equal(moved[:, [0, 1, 3, 4]], Cq[:, [0, 1, 3, 4]]) and np.array_equal(moved[:, 2], Cq[:, 2] + 9)
+    nhwc = Cq.reshape(1, 7, 1, 5)                                                          # channel-last tensors too
+    assert np.array_equal(orc.add_bias(nhwc, bias).reshape(7, 5), orc.add_bias(Cq, bias))
+    with pytest.raises(orc.OracleOverflow):
+        orc.add_bias(np.array([[2 ** 31 - 1]], np.int32), np.array([1], np.int32))
+    assert orc.add_bias(np.array([[2 ** 31 - 1]], np.int32), np.array([1], np.int32), allow_overflow=True)[0, 0] == -2 ** 31
+
+
+def test_bias_equals_one_more_k_row():
+    """A bias in the int8 range is the product with one more k: a column of ones appended to A and the bias
+    appended to every column of B -- the GEMM oracle itself says what the sum must be."""
+    rng = np.random.default_rng(6)
+    M, N, K = 9, 6, 13
+    A = rng.integers(-128, 128, size=(M, K)).astype(np.int8)
+    B = rng.integers(-128, 128, size=(N, K)).astype(np.int8)                               # row j = column j of B
+    bias = rng.integers(-128, 128, size=N).astype(np.int32)
+    A1 = np.concatenate([A, np.ones((M, 1), np.int8)], axis=1)
+    B1 = np.concatenate([B, bias.astype(np.int8).reshape(N, 1)], axis=1)
+    want = orc.gemm(A1.reshape(-1), B1.reshape(-1), M, N, K + 1).reshape(M, N)
+    got = orc.add_bias(orc.gemm(A.reshape(-1), B.reshape(-1), M, N, K).reshape(M, N), bias)
+    assert np.array_equal(got, want)
