@@ -232,6 +232,41 @@ int mipgemm_conv_u8s8f32_dequant(int64_t Nb, int64_t H, int64_t W, int64_t Cin, 
                                  float scale, void *stream);
 
 /*
+ * The fused output transforms with a per-output-channel integer bias: the exact sum of column j (GEMM)
+ * or output channel j (convolution) becomes sum + bias[j] in int32 before it is scaled, i.e.
+ * C = scale * (A * B + 1 bias^T) and C = sat8(rne(scale * (A * B + 1 bias^T))).  The paper's scheme
+ * (Section 7.3) carries a scale only; with the bias of a layer quantised at the scale s_A s_B this is
+ * the usual integer form of C^r = s_A s_B C^q + b^r, so the transform is an extension, not the paper's.
+ *
+ *   bias : device, N (GEMM) or Cout (convolution) int32 values, 4-byte aligned (16-byte aligned
+ *          reads fastest); read-only, must stay valid until the call has run on its stream.  NULL = no
+ *          bias (then the call is the entry point without the suffix).  sum + bias[j] must fit int32
+ *          (it wraps modulo 2^32 otherwise, like an accumulate that overflows).
+ * K == 0 gives the transformed bias in every row.  Everything else as for the entry points without
+ * the suffix (same rounding rules, operands, limits, errors, stream semantics).
+ */
+int mipgemm_s8s8f32_dequant_bias(int64_t M, int64_t N, int64_t K,
+                                 const int8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                                 float *C, int64_t ldc, float scale, const int32_t *bias, void *stream);
+int mipgemm_u8s8f32_dequant_bias(int64_t M, int64_t N, int64_t K,
+                                 const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                                 float *C, int64_t ldc, float scale, const int32_t *bias, void *stream);
+int mipgemm_conv_u8s8f32_dequant_bias(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int R, int S,
+                                      int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                                      const uint8_t *X, const int8_t *Wt, float *Y, float scale,
+                                      const int32_t *bias, void *stream);
+int mipgemm_s8s8s8_requant_bias(int64_t M, int64_t N, int64_t K,
+                                const int8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                                int8_t *C, int64_t ldc, float scale, int relu, const int32_t *bias, void *stream);
+int mipgemm_u8s8u8_requant_bias(int64_t M, int64_t N, int64_t K,
+                                const uint8_t *A, int64_t lda, const int8_t *B, int64_t ldb,
+                                uint8_t *C, int64_t ldc, float scale, const int32_t *bias, void *stream);
+int mipgemm_conv_u8s8u8_requant_bias(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int R, int S,
+                                     int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                                     const uint8_t *X, const int8_t *Wt, uint8_t *Y, float scale,
+                                     const int32_t *bias, void *stream);
+
+/*
  * Host-buffer variants (the end-to-end path): A, B and C are HOST pointers (pinned or
  * pageable) with the same layouts as above.  The call stages the operands into a device
  * staging buffer, runs the device entry point, copies the M x N result back into C (padding

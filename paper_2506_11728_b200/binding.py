@@ -46,6 +46,12 @@ SIGNATURES = {
     "mipgemm_s8s8s8_requant": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _int, _vp]),
     "mipgemm_u8s8u8_requant": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp]),
     "mipgemm_conv_u8s8u8_requant": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, ctypes.c_float, _vp]),
+    "mipgemm_s8s8f32_dequant_bias": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp, _vp]),
+    "mipgemm_u8s8f32_dequant_bias": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp, _vp]),
+    "mipgemm_conv_u8s8f32_dequant_bias": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, ctypes.c_float, _vp, _vp]),
+    "mipgemm_s8s8s8_requant_bias": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _int, _vp, _vp]),
+    "mipgemm_u8s8u8_requant_bias": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, ctypes.c_float, _vp, _vp]),
+    "mipgemm_conv_u8s8u8_requant_bias": (_int, [_i64] * 5 + [_int] * 8 + [_vp, _vp, _vp, ctypes.c_float, _vp, _vp]),
     "mipgemm_host_s8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_host_u8s8s32": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
     "mipgemm_s8s8s32_static_scratch": (_int, [_i64, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _int, _vp]),
@@ -166,6 +172,46 @@ def mipgemm_conv_u8s8u8_requant(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, p
     return _check(_lib.mipgemm_conv_u8s8u8_requant(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
                                                    dil_h, dil_w, _ptr(X), _ptr(Wt), _ptr(Y), float(scale),
                                                    _stream(stream)), check)
+
+
+def mipgemm_s8s8f32_dequant_bias(M, N, K, A, lda, B, ldb, C, ldc, scale, bias, stream=None, check=True) -> int:
+    """C[float32] = scale * (A * B + bias[column])."""
+    return _check(_lib.mipgemm_s8s8f32_dequant_bias(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                                    float(scale), _ptr(bias), _stream(stream)), check)
+
+
+def mipgemm_u8s8f32_dequant_bias(M, N, K, A, lda, B, ldb, C, ldc, scale, bias, stream=None, check=True) -> int:
+    """C[float32] = scale * (A * B + bias[column]), A unsigned."""
+    return _check(_lib.mipgemm_u8s8f32_dequant_bias(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                                    float(scale), _ptr(bias), _stream(stream)), check)
+
+
+def mipgemm_conv_u8s8f32_dequant_bias(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w,
+                                      X, Wt, Y, scale, bias, stream=None, check=True) -> int:
+    """Y[float32 NHWC] = scale * (Conv(Wt, X) + bias[channel])."""
+    return _check(_lib.mipgemm_conv_u8s8f32_dequant_bias(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
+                                                         dil_h, dil_w, _ptr(X), _ptr(Wt), _ptr(Y), float(scale),
+                                                         _ptr(bias), _stream(stream)), check)
+
+
+def mipgemm_s8s8s8_requant_bias(M, N, K, A, lda, B, ldb, C, ldc, scale, bias, relu=0, stream=None, check=True) -> int:
+    """C[int8] = sat(rne(scale * (A * B + bias[column]))) (clamped at 0 from below with relu)."""
+    return _check(_lib.mipgemm_s8s8s8_requant_bias(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                                   float(scale), int(bool(relu)), _ptr(bias), _stream(stream)), check)
+
+
+def mipgemm_u8s8u8_requant_bias(M, N, K, A, lda, B, ldb, C, ldc, scale, bias, stream=None, check=True) -> int:
+    """C[uint8] = sat(rne(scale * (A * B + bias[column]))), A unsigned."""
+    return _check(_lib.mipgemm_u8s8u8_requant_bias(M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                                   float(scale), _ptr(bias), _stream(stream)), check)
+
+
+def mipgemm_conv_u8s8u8_requant_bias(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w,
+                                     X, Wt, Y, scale, bias, stream=None, check=True) -> int:
+    """Y[uint8 NHWC] = sat(rne(scale * (Conv(Wt, X) + bias[channel])))."""
+    return _check(_lib.mipgemm_conv_u8s8u8_requant_bias(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w,
+                                                        dil_h, dil_w, _ptr(X), _ptr(Wt), _ptr(Y), float(scale),
+                                                        _ptr(bias), _stream(stream)), check)
 
 
 def mipgemm_s8s8f32_dequant(M, N, K, A, lda, B, ldb, C, ldc, scale, stream=None, check=True) -> int:

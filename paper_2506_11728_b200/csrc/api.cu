@@ -23,6 +23,8 @@ thread_local int tl_out_f32 = 0;
 thread_local float tl_out_scale = 1.0f;
 // ... or requantisation to 8-bit codes (the *_requant entry points): clamp bounds; C then holds bytes
 thread_local int tl_out_q8 = 0, tl_q_lo = 0, tl_q_hi = 0;
+// ... and the optional per-output-channel bias of the *_bias entry points (device pointer, length N)
+thread_local const int32_t* tl_bias = nullptr;
 
 // Experiment overrides (mipgemm_set_tuning).  The four values travel in one atomic word, so a call
 // that runs while another thread changes them sees either the old set or the new one, never a mix.
@@ -555,6 +557,7 @@ uint64_t out_mode_word() {
 
 int run_dense(DenseParams& p, const Plan& pl, long long M, long long N, int32_t* C, long long ldc,
               int accumulate, DeviceState* dev, cudaStream_t stream, bool c_map_ready = false) {
+    p.bias = tl_bias;   // (not part of the plan: a cached plan serves any bias vector)
     if (pl.split_k > 1 && !pl.cluster_split && !accumulate) {
         cudaError_t e = launch_fill_zero(C, ldc, M, N, stream);
         ++g_launches;
@@ -625,6 +628,13 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     if (st != MIPGEMM_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
 
+    if (K == 0 && tl_bias) {     // every sum is its channel's bias
+        tl_last_path = MIPGEMM_PATH_TRIVIAL | path_flags;
+        cudaError_t e = launch_bias_rows(C, ldc, M, N, tl_bias, tl_out_q8, tl_out_scale, tl_q_lo, tl_q_hi, stream);
+        ++g_launches;
+        if (e != cudaSuccess) return cuda_fail(e);
+        return MIPGEMM_OK;
+    }
     if (K == 0 && tl_out_q8) {   // every sum is 0 and so is its code (q_lo <= 0 <= q_hi)
         tl_last_path = MIPGEMM_PATH_TRIVIAL | path_flags;
         cudaError_t e = cudaMemset2DAsync(C, static_cast<size_t>(ldc), 0, static_cast<size_t>(N),
@@ -643,7 +653,7 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     }
 
     // ---- skinny path
-    if (M <= 16 && !tl_out_q8 && tun.force_path != MIPGEMM_PATH_DENSE &&
+    if (M <= 16 && !tl_out_q8 && !tl_bias && tun.force_path != MIPGEMM_PATH_DENSE &&
         tun.force_path != MIPGEMM_PATH_DENSE_PAIR) {
         SkinnyParams sp{A, lda, B, ldb, C, ldc, static_cast<int>(M), static_cast<int>(N),
                         static_cast<int>(K), a_unsigned ? 1 : 0, accumulate ? 1 : 0, tl_out_f32, tl_out_scale};
@@ -1488,6 +1498,65 @@ int mipgemm_conv_u8s8u8_requant(int64_t Nb, int64_t H, int64_t W, int64_t Cin, i
     RequantScope scope(scale, 0, 255);
     return mipgemm_conv_u8s8s32(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w, X, Wt,
                                 reinterpret_cast<int32_t*>(Y), 0, stream);
+}
+
+// The same fused transforms with a per-output-channel bias added to the exact sums first.
+struct BiasScope {
+    explicit BiasScope(const int32_t* bias) { tl_bias = bias; }
+    ~BiasScope() { tl_bias = nullptr; }
+};
+static bool bias_ok(const int32_t* bias) { return reinterpret_cast<uintptr_t>(bias) % 4 == 0; }
+
+int mipgemm_s8s8f32_dequant_bias(int64_t M, int64_t N, int64_t K, const int8_t* A, int64_t lda, const int8_t* B,
+                                 int64_t ldb, float* C, int64_t ldc, float scale, const int32_t* bias,
+                                 void* stream) {
+    if (!bias_ok(bias)) return MIPGEMM_ERR_INVALID_ARG;
+    BiasScope with_bias(bias);
+    return mipgemm_s8s8f32_dequant(M, N, K, A, lda, B, ldb, C, ldc, scale, stream);
+}
+
+int mipgemm_u8s8f32_dequant_bias(int64_t M, int64_t N, int64_t K, const uint8_t* A, int64_t lda, const int8_t* B,
+                                 int64_t ldb, float* C, int64_t ldc, float scale, const int32_t* bias,
+                                 void* stream) {
+    if (!bias_ok(bias)) return MIPGEMM_ERR_INVALID_ARG;
+    BiasScope with_bias(bias);
+    return mipgemm_u8s8f32_dequant(M, N, K, A, lda, B, ldb, C, ldc, scale, stream);
+}
+
+int mipgemm_conv_u8s8f32_dequant_bias(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int R, int S,
+                                      int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                                      const uint8_t* X, const int8_t* Wt, float* Y, float scale,
+                                      const int32_t* bias, void* stream) {
+    if (!bias_ok(bias)) return MIPGEMM_ERR_INVALID_ARG;
+    BiasScope with_bias(bias);
+    return mipgemm_conv_u8s8f32_dequant(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w,
+                                        X, Wt, Y, scale, stream);
+}
+
+int mipgemm_s8s8s8_requant_bias(int64_t M, int64_t N, int64_t K, const int8_t* A, int64_t lda, const int8_t* B,
+                                int64_t ldb, int8_t* C, int64_t ldc, float scale, int relu, const int32_t* bias,
+                                void* stream) {
+    if (!bias_ok(bias)) return MIPGEMM_ERR_INVALID_ARG;
+    BiasScope with_bias(bias);
+    return mipgemm_s8s8s8_requant(M, N, K, A, lda, B, ldb, C, ldc, scale, relu, stream);
+}
+
+int mipgemm_u8s8u8_requant_bias(int64_t M, int64_t N, int64_t K, const uint8_t* A, int64_t lda, const int8_t* B,
+                                int64_t ldb, uint8_t* C, int64_t ldc, float scale, const int32_t* bias,
+                                void* stream) {
+    if (!bias_ok(bias)) return MIPGEMM_ERR_INVALID_ARG;
+    BiasScope with_bias(bias);
+    return mipgemm_u8s8u8_requant(M, N, K, A, lda, B, ldb, C, ldc, scale, stream);
+}
+
+int mipgemm_conv_u8s8u8_requant_bias(int64_t Nb, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int R, int S,
+                                     int stride_h, int stride_w, int pad_h, int pad_w, int dil_h, int dil_w,
+                                     const uint8_t* X, const int8_t* Wt, uint8_t* Y, float scale,
+                                     const int32_t* bias, void* stream) {
+    if (!bias_ok(bias)) return MIPGEMM_ERR_INVALID_ARG;
+    BiasScope with_bias(bias);
+    return mipgemm_conv_u8s8u8_requant(Nb, H, W, Cin, Cout, R, S, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w,
+                                       X, Wt, Y, scale, stream);
 }
 
 int mipgemm_batched_s8s8s32(int64_t batch, int64_t M, int64_t N, int64_t K, const int8_t* A, int64_t lda,

@@ -134,6 +134,33 @@ cudaError_t launch_fill_zero(int32_t* C, long long ldc, long long M, long long N
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------- K == 0 with a bias
+// Every sum is its channel's bias: each row of the output is the transformed bias vector (binary32
+// scale * bias, or the clamped 8-bit code of it; same arithmetic as the dense kernel's epilogue).
+__global__ void mip_bias_rows_kernel(void* out, long long ld, long long M, long long N, const int32_t* bias,
+                                     int q8, float scale, int q_lo, int q_hi) {
+    const long long total = M * N;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long r = i / N, c = i - r * N;
+        const float t = __fmul_rn(__int2float_rn(__ldg(bias + c)), scale);
+        if (q8) {
+            const float u = fminf(fmaxf(t, static_cast<float>(q_lo)), static_cast<float>(q_hi));
+            static_cast<uint8_t*>(out)[r * ld + c] = static_cast<uint8_t>(__float2int_rn(u));
+        } else {
+            static_cast<float*>(out)[r * ld + c] = t;
+        }
+    }
+}
+
+cudaError_t launch_bias_rows(void* out, long long ld, long long M, long long N, const int32_t* bias, int q8,
+                             float scale, int q_lo, int q_hi, cudaStream_t stream) {
+    if (M <= 0 || N <= 0) return cudaSuccess;
+    const long long blocks = min((M * N + 255) / 256, 148LL * 16);
+    mip_bias_rows_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(out, ld, M, N, bias, q8, scale, q_lo, q_hi);
+    return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------- explicit im2col
 // out[m][k], m = ((n*Ho + ho)*Wo + wo), k = (r*S + s)*Cin + c; taps outside the image and
 // the pitch padding k >= k_real are zero.  One thread produces 16 consecutive k.

@@ -67,9 +67,21 @@ __device__ __forceinline__ TileCoord decode_unit(const DenseParams& p, int unit,
     return c;
 }
 
+// Optional per-output-channel int32 bias, added to the exact sums before they are scaled (an extension
+// of the paper's scale-only transform, Section 7.3).  v holds 32 consecutive columns starting at col0;
+// every lane of a warp reads the same 32 words (one broadcast request per load, served by L1).
+__device__ __forceinline__ void add_bias_chunk(const DenseParams& p, uint32_t (&v)[32], int col0) {
+    const int32_t* b = p.bias + col0;
+    const int cols = p.N - col0;
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+        if (j < cols) v[j] += static_cast<uint32_t>(__ldg(b + j));
+}
+
 // Fused dequantisation (paper Section 7.3, C^r = s_A s_B C^q): the exact int32 sum is converted to
 // binary32 (round to nearest even) and multiplied by the scale in binary32.
-__device__ __forceinline__ void dequant_chunk(const DenseParams& p, uint32_t (&v)[32]) {
+__device__ __forceinline__ void dequant_chunk(const DenseParams& p, uint32_t (&v)[32], int col0) {
+    if (p.bias) add_bias_chunk(p, v, col0);
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__int2float_rn(static_cast<int>(v[j])) * p.out_scale);
 }
@@ -899,10 +911,12 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     for (; c0 < n_here; c0 += 2 * step) {
                         tmem_ld_wait();
                         if (c0 + step < n_here) tmem_ld_32x32(t_row + c0 + step, vb);
+                        if (p.bias) add_bias_chunk(p, va, tc.n0 + c0);
                         if (row < p.M) store_q8_chunk(p, crow8 + c0, va, min(32, n_here - c0));
                         if (c0 + step < n_here) {
                             tmem_ld_wait();
                             if (c0 + 2 * step < n_here) tmem_ld_32x32(t_row + c0 + 2 * step, va);
+                            if (p.bias) add_bias_chunk(p, vb, tc.n0 + c0 + step);
                             if (row < p.M) store_q8_chunk(p, crow8 + c0 + step, vb, min(32, n_here - c0 - step));
                         }
                     }
@@ -911,7 +925,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     for (int c0 = 0; c0 < n_here; c0 += 32) {
                         tmem_ld_32x32(t_row + c0, va);
                         tmem_ld_wait();
-                        if (p.out_f32) dequant_chunk(p, va);
+                        if (p.out_f32) dequant_chunk(p, va, tc.n0 + c0);
                         if (p.c_mode == 1) tma_store_slab(p, staging + (chunk_no & 1u) * 16384u, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
                         else if (p.c_mode == 3) coalesced_chunk(p, my_staging + (chunk_no & 1u) * 4096u, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
                         else if (p.c_mode == 5) rows_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
@@ -929,7 +943,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { p.trace[57] += clock64() - tw0; p.trace[58] += 1; }
 #endif
                     if (c0 + 32 < n_here) tmem_ld_32x32(t_row + c0 + 32, vb);
-                    if (p.out_f32) dequant_chunk(p, va);
+                    if (p.out_f32) dequant_chunk(p, va, tc.n0 + c0);
                     if (p.c_mode == 1) tma_store_slab(p, staging + (chunk_no & 1u) * 16384u, va, lane, q, warp == 2, tc.n0 + c0, m_cta, tc.batch);
                     else if (p.c_mode == 3) coalesced_chunk(p, my_staging, va, lane, m_cta + q * 32, tc.n0 + c0, c_off);
                     else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + (chunk_no & 1u) * 4096u, va, lane, tc.n0 + c0, m_cta + q * 32);
@@ -939,7 +953,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     if (c0 + 32 < n_here) {
                         tmem_ld_wait();
                         if (c0 + 64 < n_here) tmem_ld_32x32(t_row + c0 + 64, va);
-                        if (p.out_f32) dequant_chunk(p, vb);
+                        if (p.out_f32) dequant_chunk(p, vb, tc.n0 + c0 + 32);
                         if (p.c_mode == 1) tma_store_slab(p, staging + (chunk_no & 1u) * 16384u, vb, lane, q, warp == 2, tc.n0 + c0 + 32, m_cta, tc.batch);
                         else if (p.c_mode == 3) coalesced_chunk(p, my_staging + 4096u, vb, lane, m_cta + q * 32, tc.n0 + c0 + 32, c_off);
                         else if (p.c_mode == 2) tma_reduce_chunk(p, my_staging + (chunk_no & 1u) * 4096u, vb, lane, tc.n0 + c0 + 32, m_cta + q * 32);
@@ -1026,7 +1040,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                         for (int e = 0; e < 4; ++e) v[4 * j + e] += x[e];
                     }
                 }
-                if (p.out_f32) dequant_chunk(p, v);
+                if (p.out_f32) dequant_chunk(p, v, col0);
                 if (p.c_mode == 1) tma_store_slab(p, staging + (c & 1) * 16384u, v, lane, q, warp == 2, col0, m_cta);
                 else if (p.c_mode == 3) coalesced_chunk(p, my_staging + (c & 1) * 4096u, v, lane, m_cta + q * 32, col0);
                 else if (row < p.M) store_chunk(p, p.C + static_cast<long long>(row) * p.ldc + col0, v, min(32, p.N - col0));

@@ -75,6 +75,7 @@ struct alignas(64) DenseParams {
     float out_scale;
     int out_q8;              // 1: the epilogue writes 8-bit codes min(max(rne(scale * sum), q_lo), q_hi); C and ldc
     int q_lo, q_hi;          //    then address bytes (c_mode 4)
+    const int32_t* bias;     // optional, length N: added to the exact sums before the output transform
     int c_mode;              // 5: rows through shared memory, 4-byte accesses (C only 4-byte aligned); 4: 8-bit codes,
                              // row-per-thread; 0: row-per-thread stores (any alignment), 1: coalesced stores through
                              // shared memory, 2: TMA tile reduce-add (split-K); 1 and 2 need a 16-byte
@@ -164,6 +165,8 @@ cudaError_t launch_transpose_repack(const void* src, long long src_pitch, void* 
 cudaError_t launch_weight_slots(const int8_t* src, int8_t* dst, long long rows, int R, int seg, int slot,
                                 cudaStream_t stream);
 cudaError_t launch_fill_zero(int32_t* C, long long ldc, long long M, long long N, cudaStream_t stream);
+cudaError_t launch_bias_rows(void* out, long long ld, long long M, long long N, const int32_t* bias, int q8,
+                             float scale, int q_lo, int q_hi, cudaStream_t stream);
 struct Im2colParams {
     const uint8_t* X; uint8_t* out;
     long long Nb, H, W, Cin, Ho, Wo;
