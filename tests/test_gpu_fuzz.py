@@ -182,6 +182,42 @@ def test_fuzz_conv(mg):
             i, X.shape, R, S, stride, pad, dil, Cout, acc, path, first_mismatch(got, want))
 
 
+def test_fuzz_conv_scaled_outputs_with_bias(mg):
+    """Random convolution geometries through the fused transforms, every other case with a per-channel bias."""
+    rng = np.random.default_rng(2031)
+    for i in range(CASES):
+        Cin = int(rng.choice([1, 3, 16, 64, 128]))
+        R, S = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        pad = (int(rng.integers(0, 2)), int(rng.integers(0, 2)))
+        stride = (int(rng.integers(1, 3)), int(rng.integers(1, 3)))
+        H, W = int(rng.integers(R, 20)), int(rng.integers(S, 20))
+        Nb = int(rng.integers(1, 4)) if rng.integers(4) else int(rng.integers(16, 120))
+        Cout = int(rng.choice([4, 7, 32, 64, 100]))
+        X = inputs.uniform_u8(Nb * H * W * Cin, 17000 + i).reshape(Nb, H, W, Cin)
+        Wt = inputs.normal_s8(Cout * R * S * Cin, 18000 + i, 32.0, -127, 127).reshape(Cout, R, S, Cin)
+        sums = orc.conv(X, Wt, stride=stride, pad=pad)
+        dbias = None
+        if rng.integers(2):
+            bias = rng.integers(-100000, 100001, size=Cout, dtype=np.int64).astype(np.int32)
+            sums = orc.add_bias(sums, bias)
+            dbias, _k = to_dev(bias, int(rng.choice([0, 4])))
+        scale = float(np.float32(255.0 / (4.0 * 32.0 * 147.0 * np.sqrt(R * S * Cin))))
+        dX, _x = to_dev(X)
+        dW, _w = to_dev(Wt)
+        dY, _y = to_dev(np.full(sums.size, 0x5A, np.uint8))
+        geo = (Nb, H, W, Cin, Cout, R, S, stride[0], stride[1], pad[0], pad[1], 1, 1)
+        mg.mipgemm_conv_u8s8u8_requant_bias(*geo, dX, dW, dY, scale, dbias)
+        assert mg.mipgemm_device_status() == mg.OK
+        want = orc.requant(sums, scale, 0, 255)
+        got = dY.cpu().numpy().reshape(sums.shape).astype(np.int32)
+        assert np.array_equal(got, want), "conv requant case %d %s f%dx%d cout %d bias %s" % (i, X.shape, R, S, Cout, dbias is not None)
+        dF, _f = to_dev(np.zeros(sums.size, np.float32))
+        mg.mipgemm_conv_u8s8f32_dequant_bias(*geo, dX, dW, dF, scale, dbias)
+        assert mg.mipgemm_device_status() == mg.OK
+        rule = (sums.astype(np.float32) * np.float32(scale)).astype(np.float32)
+        assert np.array_equal(dF.cpu().numpy().view(np.float32).reshape(sums.shape), rule), "conv dequant case %d" % i
+
+
 def test_fuzz_scaled_outputs(mg):
     rng = np.random.default_rng(2027)
     for i in range(CASES):
@@ -193,16 +229,22 @@ def test_fuzz_scaled_outputs(mg):
         scale = float(np.float32(rng.choice([1.0, 0.5, 2.0 ** -7, 1.3e-3, 7.7e-5]) * (1 if rng.integers(2) else -1)))
         dA, _a = to_dev(A)
         dB, _b = to_dev(B)
+        # every other case with a per-column bias (its pointer 4-, 8- or 16-byte aligned)
+        dbias = None
+        if rng.integers(2):
+            bias = rng.integers(-200000, 200001, size=N, dtype=np.int64).astype(np.int32)
+            sums = orc.add_bias(sums, bias)
+            dbias, _k = to_dev(bias, int(rng.choice([0, 4, 8])))
         # 8-bit codes
         ldc = N + int(rng.choice([0, 3, 16]))
         dC, _c = to_dev(np.full(M * ldc, 0x5A, np.uint8), int(rng.choice([0, 1])))
         if unsigned:
-            mg.mipgemm_u8s8u8_requant(M, N, K, dA, K, dB, K, dC, ldc, scale)
+            mg.mipgemm_u8s8u8_requant_bias(M, N, K, dA, K, dB, K, dC, ldc, scale, dbias)
             want = orc.requant(sums, scale, 0, 255)
             got = dC.cpu().numpy().reshape(M, ldc)[:, :N].astype(np.int32)
         else:
             relu = int(rng.integers(2))
-            mg.mipgemm_s8s8s8_requant(M, N, K, dA, K, dB, K, dC, ldc, scale, relu)
+            mg.mipgemm_s8s8s8_requant_bias(M, N, K, dA, K, dB, K, dC, ldc, scale, dbias, relu)
             want = orc.requant(sums, scale, 0 if relu else -128, 127)
             got = dC.cpu().numpy().reshape(M, ldc)[:, :N].view(np.int8).astype(np.int32)
         assert mg.mipgemm_device_status() == mg.OK
@@ -210,7 +252,8 @@ def test_fuzz_scaled_outputs(mg):
         assert (dC.cpu().numpy().reshape(M, ldc)[:, N:] == 0x5A).all()
         # float32
         dF, _f = to_dev(np.zeros(M * N, np.float32))
-        (mg.mipgemm_u8s8f32_dequant if unsigned else mg.mipgemm_s8s8f32_dequant)(M, N, K, dA, K, dB, K, dF, N, scale)
+        (mg.mipgemm_u8s8f32_dequant_bias if unsigned else mg.mipgemm_s8s8f32_dequant_bias)(M, N, K, dA, K, dB, K, dF, N,
+                                                                                         scale, dbias)
         gotf = dF.cpu().numpy().view(np.float32).reshape(M, N)
         rule = (sums.astype(np.float32) * np.float32(scale)).astype(np.float32)
         assert np.array_equal(gotf, rule), "dequant case %d" % i
