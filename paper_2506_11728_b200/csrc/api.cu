@@ -470,7 +470,9 @@ void fill_common(DenseParams& p, const Plan& pl, long long M, long long N, int32
                 p.use_red = 0;
             }
         } else {
-            p.c_mode = (accumulate || !tma_ok) ? 3 : 1;
+            // (accumulate: the tile stores become tile reduce-adds; without tile stores the rows are added
+            // element-wise at the L2, which beats reading, adding and writing 16-byte pieces)
+            p.c_mode = tma_ok ? 1 : (accumulate ? 5 : 3);
         }
     }
     // A C that is only 4-byte aligned: rows through shared memory, one 128-byte run per store instruction

@@ -208,8 +208,14 @@ __device__ __forceinline__ void tma_store_slab(const DenseParams& p, uint32_t bu
     const long long ts5 = clock64();
 #endif
     if (issuer && elect_one()) {
-        if (p.batch > 1) tma_store_3d(&p.tmap_c, buf, x, y, z);
-        else tma_store_2d(&p.tmap_c, buf, x, y);
+        if (p.accumulate) {   // C += : the slab is added to C at the L2 (32-bit integer adds, exact in any order)
+            if (p.batch > 1) tma_reduce_add_3d(&p.tmap_c, buf, x, y, z);
+            else tma_reduce_add_2d(&p.tmap_c, buf, x, y);
+        } else if (p.batch > 1) {
+            tma_store_3d(&p.tmap_c, buf, x, y, z);
+        } else {
+            tma_store_2d(&p.tmap_c, buf, x, y);
+        }
         tma_store_commit();
     }
 #ifdef MIPGEMM_TRACE
@@ -347,19 +353,15 @@ __device__ __forceinline__ void rows_chunk(const DenseParams& p, uint32_t buf, c
         }
         return;
     }
-    // all loads of the incoming C first: 32 independent accesses in flight instead of 32 round trips
-    uint32_t c[32];
-#pragma unroll
-    for (int r = 0; r < 32; ++r) c[r] = r < rows ? static_cast<uint32_t>(dst[static_cast<long long>(r) * p.ldc]) : 0u;
-#pragma unroll
-    for (int r = 0; r < 32; ++r) {
-        if (r < rows) {
-            uint32_t x;
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(x)
-                         : "r"(buf + static_cast<uint32_t>(r) * 128u + (static_cast<uint32_t>((lane >> 2) ^ (r & 7)) << 4) +
-                               static_cast<uint32_t>(lane & 3) * 4u) : "memory");
-            dst[static_cast<long long>(r) * p.ldc] = static_cast<int32_t>(x + c[r]);
-        }
+    // C += : the sums are added at the L2 (32-bit integer reductions, one 128-byte run per instruction): exact in
+    // any order, and no thread waits for the old value of C
+    for (int r = 0; r < rows; ++r) {
+        uint32_t x;
+        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(x)
+                     : "r"(buf + static_cast<uint32_t>(r) * 128u + (static_cast<uint32_t>((lane >> 2) ^ (r & 7)) << 4) +
+                           static_cast<uint32_t>(lane & 3) * 4u) : "memory");
+        red_add_s32(dst, x);
+        dst += p.ldc;
     }
 }
 
@@ -1043,6 +1045,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 if (p.out_f32) dequant_chunk(p, v, col0);
                 if (p.c_mode == 1) tma_store_slab(p, staging + (c & 1) * 16384u, v, lane, q, warp == 2, col0, m_cta);
                 else if (p.c_mode == 3) coalesced_chunk(p, my_staging + (c & 1) * 4096u, v, lane, m_cta + q * 32, col0);
+                else if (p.c_mode == 5) rows_chunk(p, my_staging + (c & 1) * 4096u, v, lane, m_cta + q * 32, col0, 0);
                 else if (row < p.M) store_chunk(p, p.C + static_cast<long long>(row) * p.ldc + col0, v, min(32, p.N - col0));
             }
             if (p.c_mode == 1 && warp == 2 && elect_one()) tma_store_wait<0>();

@@ -52,7 +52,7 @@ constexpr int kSmemBudget = 227 * 1024;
 struct alignas(64) DenseParams {
     CUtensorMap tmap_a;      // tiled {K, M} byte tensor, or im2col-mode NHWC tensor
     CUtensorMap tmap_b;      // tiled {K, N} byte tensor (weights, K contiguous)
-    CUtensorMap tmap_c;      // tiled {N, M} int32 tensor, 32 x 32 boxes (used when c_mode == 2)
+    CUtensorMap tmap_c;      // tiled {N, M} int32 tensor: 32 x 128 boxes (c_mode 1) or 32 x 32 boxes (c_mode 2)
     int32_t* C;
     long long ldc;
     int M, N;
@@ -76,10 +76,12 @@ struct alignas(64) DenseParams {
     int out_q8;              // 1: the epilogue writes 8-bit codes min(max(rne(scale * sum), q_lo), q_hi); C and ldc
     int q_lo, q_hi;          //    then address bytes (c_mode 4)
     const int32_t* bias;     // optional, length N: added to the exact sums before the output transform
-    int c_mode;              // 5: rows through shared memory, 4-byte accesses (C only 4-byte aligned); 4: 8-bit codes,
-                             // row-per-thread; 0: row-per-thread stores (any alignment), 1: coalesced stores through
-                             // shared memory, 2: TMA tile reduce-add (split-K); 1 and 2 need a 16-byte
-                             // aligned C base and ldc % 4 == 0
+    int c_mode;              // 0: row-per-thread stores (any alignment); 1: TMA tile stores of 128 x 32 slabs -- tile
+                             // reduce-adds when `accumulate` is set; 2: TMA tile reduce-add of 32 x 32 boxes (explicit
+                             // split-K); 3: 16-byte pieces through a transposing shared-memory buffer; 4: 8-bit codes,
+                             // row-per-thread; 5: rows through shared memory, 4-byte accesses, one 128-byte run per
+                             // instruction (any alignment; `accumulate` adds at the L2 with red.global.add).
+                             // 1, 2 and 3 need a 16-byte aligned C base and ldc % 4 == 0, 1 and 2 also N % 4 == 0
     uint32_t idesc;          // tcgen05 instruction descriptor
     uint32_t tmem_cols;      // power of two >= 2*block_n
     // implicit im2col (operand A gathered by TMA im2col loads)
