@@ -156,7 +156,7 @@ def build_ragged(torch, mg):
     p = _gemm_problem(torch, mg, "ragged_1000x3001x777_acc", M, N, K, A, B, C0=C0, sets=10)
     return Workload("ragged", [p], "TOPS", "int8_gemm_tops",
                     "s8*s8->s32 M,N,K = 1000,3001,777, every pitch misaligned, accumulate=1 onto a seeded int32 C",
-                    "hbm", "mip_dense_kernel (+ 2 re-pitch launches)",
+                    "hbm", "mip_dense_kernel (+ 1 re-pitch launch for both operands)",
                     "10 copies of the 27 MB problem used in turn (270 MB > L2)")
 
 

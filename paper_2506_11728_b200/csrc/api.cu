@@ -748,7 +748,17 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
     const void* a_use = A;
     const void* b_use = B;
     long long lda_use = lda, ldb_use = ldb;
-    if (repack_a) {
+    if (repack_a && repack_b) {   // both operands in one launch
+        void* dst_a = scratch.take(static_cast<size_t>(M) * pitch);
+        void* dst_b = scratch.take(static_cast<size_t>(N) * pitch);
+        cudaError_t e = launch_repack2(A, lda, dst_a, M, B, ldb, dst_b, N, pitch, K, stream);
+        ++g_launches;
+        if (e != cudaSuccess) return cuda_fail(e);
+        a_use = dst_a;
+        b_use = dst_b;
+        lda_use = ldb_use = pitch;
+        path_flags |= MIPGEMM_PATH_REPACK;
+    } else if (repack_a) {
         void* dst = scratch.take(static_cast<size_t>(M) * pitch);
         cudaError_t e = launch_repack(A, lda, dst, pitch, M, K, stream);
         ++g_launches;
@@ -757,7 +767,7 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
         lda_use = pitch;
         path_flags |= MIPGEMM_PATH_REPACK;
     }
-    if (repack_b) {
+    if (repack_b && !repack_a) {
         void* dst = scratch.take(static_cast<size_t>(N) * pitch);
         cudaError_t e = launch_repack(B, ldb, dst, pitch, N, K, stream);
         ++g_launches;

@@ -11,14 +11,23 @@ namespace mip {
 // dst[r][0..cols) = src[r][0..cols); dst is 16-byte aligned with a pitch that is a
 // multiple of 16, src has byte alignment only.  Each thread assembles 16 bytes from
 // aligned 32-bit words; only words holding at least one valid byte are read.
-__global__ void mip_repack_kernel(const uint8_t* __restrict__ src, long long src_pitch,
-                                  uint8_t* __restrict__ dst, long long dst_pitch,
-                                  long long rows, long long chunks_per_row, long long cols) {
-    const long long total = rows * chunks_per_row;
+// One launch serves up to two matrices with the same number of columns (both operands of a GEMM): chunks
+// [0, rows0 * chunks_per_row) belong to the first, the rest to the second.
+__global__ void mip_repack_kernel(const uint8_t* __restrict__ src0, long long src_pitch0, uint8_t* __restrict__ dst0,
+                                  long long rows0, const uint8_t* __restrict__ src1, long long src_pitch1,
+                                  uint8_t* __restrict__ dst1, long long rows1, long long dst_pitch,
+                                  long long chunks_per_row, long long cols) {
+    const long long total0 = rows0 * chunks_per_row;
+    const long long total = total0 + rows1 * chunks_per_row;
     for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
          i += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const long long r = i / chunks_per_row;
-        const long long c = (i - r * chunks_per_row) * 16;
+        const bool second = i >= total0;
+        const uint8_t* src = second ? src1 : src0;
+        uint8_t* dst = second ? dst1 : dst0;
+        const long long src_pitch = second ? src_pitch1 : src_pitch0;
+        const long long ii = second ? i - total0 : i;
+        const long long r = ii / chunks_per_row;
+        const long long c = (ii - r * chunks_per_row) * 16;
         const int nvalid = static_cast<int>(min(16LL, cols - c));
         const uint8_t* s = src + r * src_pitch + c;
         const unsigned off = static_cast<unsigned>(reinterpret_cast<uintptr_t>(s) & 3u);
@@ -36,17 +45,23 @@ __global__ void mip_repack_kernel(const uint8_t* __restrict__ src, long long src
     }
 }
 
-cudaError_t launch_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,
-                          long long rows, long long cols, cudaStream_t stream) {
-    if (rows <= 0 || cols <= 0) return cudaSuccess;
+cudaError_t launch_repack2(const void* src0, long long src_pitch0, void* dst0, long long rows0, const void* src1,
+                           long long src_pitch1, void* dst1, long long rows1, long long dst_pitch, long long cols,
+                           cudaStream_t stream) {
+    if (rows0 + rows1 <= 0 || cols <= 0) return cudaSuccess;
     const long long chunks = (cols + 15) / 16;
-    const long long total = rows * chunks;
+    const long long total = (rows0 + rows1) * chunks;
     const int threads = 256;
     const long long blocks = min((total + threads - 1) / threads, 148LL * 16);
     mip_repack_kernel<<<static_cast<unsigned>(blocks), threads, 0, stream>>>(
-        static_cast<const uint8_t*>(src), src_pitch, static_cast<uint8_t*>(dst), dst_pitch, rows,
-        chunks, cols);
+        static_cast<const uint8_t*>(src0), src_pitch0, static_cast<uint8_t*>(dst0), rows0,
+        static_cast<const uint8_t*>(src1), src_pitch1, static_cast<uint8_t*>(dst1), rows1, dst_pitch, chunks, cols);
     return cudaGetLastError();
+}
+
+cudaError_t launch_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,
+                          long long rows, long long cols, cudaStream_t stream) {
+    return launch_repack2(src, src_pitch, dst, rows, nullptr, 0, nullptr, 0, dst_pitch, cols, stream);
 }
 
 // ---------------------------------------------------------------- transposing repack

@@ -161,6 +161,9 @@ cudaError_t launch_skinny_ring16(const SkinnyRingParams& p, int sm_count, cudaSt
 // Auxiliary kernels.
 cudaError_t launch_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,
                           long long rows, long long cols, cudaStream_t stream);
+cudaError_t launch_repack2(const void* src0, long long src_pitch0, void* dst0, long long rows0, const void* src1,
+                           long long src_pitch1, void* dst1, long long rows1, long long dst_pitch, long long cols,
+                           cudaStream_t stream);
 cudaError_t launch_transpose_repack(const void* src, long long src_pitch, void* dst, long long dst_pitch,
                                     long long rows_out, long long cols_out, cudaStream_t stream);
 // Weights [rows][R][seg] -> [rows][R][slot], zero padded (slot >= seg, slot % 16 == 0).
