@@ -988,7 +988,7 @@ def main():
     cpu = None
     if want_cpu:
         from oracle import mip_oracle as orc
-        frac = calibrate_fraction(wl.probs, 15.0)
+        frac = calibrate_fraction(wl.probs, 24.0)
         gpu_rows = {}
         for p, r in zip(wl.probs, oracle_sample_rows(wl.probs, frac)):
             gpu_rows[p.name] = p.bufs[2][:r * p.dims[1]].cpu().numpy()
