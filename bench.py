@@ -662,8 +662,7 @@ def parity_workload(torch, wl, rows_per_problem=48):
             t_or += time.perf_counter() - t0
             if p.accumulate:   # the buffer has received the product once per launch since it held C0
                 total = C0.reshape(M, ldc)[rows, :N].astype(np.int64) + wl.steps_run * want.astype(np.int64)
-                assert np.abs(total).max() < 2 ** 31
-                want = total.astype(np.int32)
+                want = (total & 0xFFFFFFFF).astype(np.uint32).view(np.int32)     # (C += wraps modulo 2^32, as documented)
         elif p.kind == "conv":
             batch, H, W, Cin, Cout, R, S, st, pd, Ho, Wo = p.geom
             X, Wt, _ = p.host
