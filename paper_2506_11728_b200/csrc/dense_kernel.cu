@@ -219,7 +219,7 @@ __device__ __forceinline__ void tma_store_slab(const DenseParams& p, uint32_t bu
         tma_store_commit();
     }
 #ifdef MIPGEMM_TRACE
-    if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) {
+    if (p.trace && (p.debug_flags & 128) && blockIdx.x == 0 && threadIdx.x == 64) {   // (perturbs: on request only)
         p.trace[50] += ts1 - ts0; p.trace[51] += ts2 - ts1; p.trace[52] += ts3 - ts2; p.trace[53] += ts4 - ts3;
         p.trace[54] += ts5 - ts4; p.trace[55] += clock64() - ts5; p.trace[56] += 1;
     }
@@ -591,14 +591,32 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             const uint32_t k_steps = p.block_k / 32;
             bool ok = true;
             int t = 0;
+#ifdef MIPGEMM_TRACE
+            // (trace builds: waits and issue time of CTA 0's MMA warp, summed in registers and written once)
+            long long acc_tempty = 0, acc_full = 0, n_tempty = 0, n_full = 0, acc_issue = 0;
+            const long long role_t0 = clock64();
+#endif
             for (int unit = first_unit; unit < total_units && ok; unit += unit_stride, ++t) {
                 const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
                 const uint32_t acc = t & 1, acc_phase = (t >> 1) & 1;
+#ifdef MIPGEMM_TRACE
+                long long tm0 = clock64();
+#endif
                 if (!mbar_wait<kPair>(bar_tempty + 8u * acc, acc_phase ^ 1u, abort_flag, budget)) { ok = false; break; }
+#ifdef MIPGEMM_TRACE
+                acc_tempty += clock64() - tm0; ++n_tempty;
+#endif
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * p.block_n;
                 for (int kb = tc.kb_begin; kb < tc.kb_end; ++kb) {
+#ifdef MIPGEMM_TRACE
+                    tm0 = clock64();
+#endif
                     if (!mbar_wait(bar_full + 8u * s, phase, abort_flag, budget)) { ok = false; break; }
+#ifdef MIPGEMM_TRACE
+                    acc_full += clock64() - tm0; ++n_full;
+                    const long long ti0 = clock64();
+#endif
                     if (t == 0 && kb == tc.kb_begin) MIP_STAMP(3);
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + s * stage_bytes;
@@ -623,6 +641,10 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                             mma_commit(empty_local);
                         }
                     }
+#ifdef MIPGEMM_TRACE
+                    __syncwarp();
+                    acc_issue += clock64() - ti0;
+#endif
                     if (++s == static_cast<uint32_t>(p.stages)) { s = 0; phase ^= 1u; }
                 }
                 if (t == 0) MIP_STAMP(4);
@@ -639,6 +661,12 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                     }
                 }
             }
+#ifdef MIPGEMM_TRACE
+            if (p.trace && blockIdx.x == 0 && lane == 0) {
+                p.trace[32] = acc_tempty; p.trace[33] = n_tempty; p.trace[34] = acc_full; p.trace[35] = n_full;
+                p.trace[36] = clock64() - role_t0; p.trace[37] = acc_issue;
+            }
+#endif
         }
     } else if (kGather && warp >= kGatherFirstWarp) {
         // ------------------------------------------------------------ software im2col
@@ -873,6 +901,11 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
         // otherwise hand the same buffer to two consecutive copies, the second overwriting what the first may
         // still be reading.
         uint32_t chunk_no = 0;
+#ifdef MIPGEMM_TRACE
+        // (trace builds: CTA 0's first epilogue warp, summed in registers and written once)
+        long long acc_e_wait = 0, acc_e_body = 0, n_e_tiles = 0;
+        const long long e_role_t0 = clock64();
+#endif
         for (int unit = first_unit; unit < total_units; unit += unit_stride, ++t) {
             const TileCoord tc = decode_unit(p, unit, kRowsPerTile);
             const uint32_t acc = t & 1, acc_phase = (t >> 1) & 1;
@@ -885,7 +918,8 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
             if (p.c_mode == 1 && p.cluster_split <= 1) gave_up = named_bar_or(1, 128, gave_up);
             if (gave_up) break;
 #ifdef MIPGEMM_TRACE
-            if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { p.trace[59] += clock64() - tt0; p.trace[60] += 1; }
+            const long long tt1 = clock64();
+            acc_e_wait += tt1 - tt0; ++n_e_tiles;
 #endif
             if (t == 0 && warp == 2) MIP_STAMP(5);
             tc_fence_after();
@@ -942,7 +976,7 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
 #endif
                     tmem_ld_wait();
 #ifdef MIPGEMM_TRACE
-                    if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { p.trace[57] += clock64() - tw0; p.trace[58] += 1; }
+                    if (p.trace && (p.debug_flags & 128) && blockIdx.x == 0 && threadIdx.x == 64) { p.trace[57] += clock64() - tw0; p.trace[58] += 1; }
 #endif
                     if (c0 + 32 < n_here) tmem_ld_32x32(t_row + c0 + 32, vb);
                     if (p.out_f32) dequant_chunk(p, va, tc.n0 + c0);
@@ -973,7 +1007,15 @@ mip_dense_kernel(const __grid_constant__ DenseParams p) {
                 if (kPair && !leader) mbar_arrive_remote(bar_tempty + 8u * acc, 0);
                 else mbar_arrive(bar_tempty + 8u * acc);
             }
+#ifdef MIPGEMM_TRACE
+            acc_e_body += clock64() - tt1;
+#endif
         }
+#ifdef MIPGEMM_TRACE
+        if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) {
+            p.trace[59] = acc_e_wait; p.trace[60] = n_e_tiles; p.trace[61] = acc_e_body; p.trace[62] = clock64() - e_role_t0;
+        }
+#endif
         // every tile copy issued by this warp must be complete before the CTA may exit
         if (p.cluster_split <= 1 && (p.c_mode == 2 || (p.c_mode == 1 && warp == 2)) && elect_one())
             tma_store_wait<0>();
