@@ -337,14 +337,14 @@ double plan_cost_us(int pair, int bn, int split, long long M, long long N, int k
     return 3.7 + (pair ? 1.0 : 0.0) + clk / 1900.0;   // pairs: cluster launch, two cluster barriers
 }
 
-Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceState* dev, int min_bn = 64,
+Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceState* dev, int min_bn = 32,
                int min_bn_pair = 64, bool one_cta_no_split = false) {
     const int sm_count = dev->sm_count;
     const Tuning tun = tuning_now();
     Plan pl{};
     pl.k_blocks = static_cast<int>((K + block_k - 1) / block_k);
 
-    // Candidates: one CTA per tile or CTA pairs, bn in {64, 128, 256}, optionally a cluster
+    // Candidates: one CTA per tile or CTA pairs, bn a multiple of 32 up to 256, optionally a cluster
     // split-K of 2/4/8 when the tiles alone would leave most SMs idle.  Experiment overrides
     // (mipgemm_set_tuning) restrict the candidate set.
     int best_pair = 0, best_bn = 128, best_split = 1;
@@ -357,9 +357,14 @@ Plan make_plan(long long M, long long N, long long K, int block_k, const DeviceS
         if (pair && (dev->pair_clusters <= 0 || one_cta_no_split)) continue;
         if (tun.force_path == MIPGEMM_PATH_DENSE_PAIR && !pair && dev->pair_clusters > 0) continue;
         if (tun.force_path == MIPGEMM_PATH_DENSE && pair) continue;
-        for (int bn = 64; bn <= 256; bn += 32) {      // any multiple of 32 columns is a legal tile width
+        for (int bn = 32; bn <= 256; bn += 32) {      // any multiple of 32 columns is a legal tile width (32 itself
+                                                      // only pays for problems of a single wave: 512^3 -7 %)
             int bn_use = bn;
             if (bn < (pair ? min_bn_pair : min_bn)) continue;
+            // (32 columns: only short-K problems that leave half of the SMs idle even at 64; K-heavy ones split K)
+            if (bn == 32 && !forced_bn &&
+                (((M + kBlockM - 1) / kBlockM) * ((N + 63) / 64) > sm_count / 2 || pl.k_blocks > 8))
+                continue;
             if (min_bn >= 128 && bn % 128 != 0) continue;   // (N-contiguous B: whole 128-column blocks)
             if (forced_bn) {
                 if (bn != 256) continue;                      // a single candidate: the forced width
