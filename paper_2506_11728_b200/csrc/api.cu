@@ -709,6 +709,7 @@ int gemm_impl(bool a_unsigned, int64_t M, int64_t N, int64_t K, const void* A, i
                                  inside_constant_range(B, static_cast<size_t>(N - 1) * ldb + K)) ? 1 : 0;
                 rp.status = dev->status_word;
                 rp.wait_budget_ns = g_wait_budget_ns.load(std::memory_order_relaxed);
+                rp.prefetch_chunks = MIP_ENV_KNOB("MIPGEMM_PREFETCH_CHUNKS", 4);   // (swept 0..16: 4 is the best)
                 rp.debug_flags = g_debug_flags.load(std::memory_order_relaxed) |
                                  (MIP_ENV_KNOB("MIPGEMM_RING_ALWAYS_RELEASE", 0) ? 2 : 0);   // (A/B switch)
                 rp.trace = nullptr;

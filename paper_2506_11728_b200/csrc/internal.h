@@ -145,6 +145,7 @@ struct alignas(64) SkinnyRingParams {
     int pdl_mode;                // 1: launched with programmatic stream serialisation (filled in by the launcher)
     int b_constant;              // 1: B may be fetched before the previous kernel on the stream has completed
     int slots, tokens_in_smem;   // filled in by the launcher
+    int prefetch_chunks;         // 16 KB chunks of B each CTA asks the L2 for before the dependency wait (no promise)
     unsigned int* status;
     unsigned long long wait_budget_ns;
     int debug_flags;             // test hook (mipgemm_debug_set): bit 0 = the first CTA never loads its second chunk

@@ -99,12 +99,20 @@ mip_skinny_ring16_kernel(const __grid_constant__ SkinnyRingParams p) {
     // complete -- except the weight producer when the caller has promised constant weights.
     __syncthreads();
     if (p.pdl_mode == 1) pdl_launch_dependents();
-    if (!(p.b_constant && warp == kConsumers)) pdl_wait();
-
     const int units = (p.N + 15) >> 4;
     const int chunks = (p.K + 1023) >> 10;
     const int my_units = (units - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
     const uint64_t budget = p.wait_budget_ns;
+    // (B is not read before the previous kernel has completed unless the caller promised constant weights, but
+    // the L2 may be asked to fetch the first chunks: a prefetch brings no data to the SM and the L2 stays coherent)
+    if (p.pdl_mode == 1 && !p.b_constant && warp == kConsumers && elect_one()) {
+        int asked = 0;
+        const int n_u = min(kMaxU, my_units);
+        for (int ch = 0; ch < chunks && asked < p.prefetch_chunks; ++ch)
+            for (int j = 0; j < n_u && asked < p.prefetch_chunks; ++j, ++asked)
+                tma_prefetch_l2_3d(&p.tmap_b, 0, (static_cast<int>(blockIdx.x) + j * static_cast<int>(gridDim.x)) * 16, ch * 8);
+    }
+    if (!(p.b_constant && warp == kConsumers)) pdl_wait();
 
     if (warp == kConsumers) {
         // ------------------------------------------------------------ weight producer

@@ -143,12 +143,23 @@ mip_skinny_ring_kernel(const __grid_constant__ SkinnyRingParams p) {
     __syncthreads();
     if (p.pdl_mode == 1) pdl_launch_dependents();
     if (warp == 0) RING_STAMP(1);
-    if (!(p.b_constant && warp == kRingConsumers)) pdl_wait();
-    if (warp == 0) RING_STAMP(2);
-
     const int units = (p.N + 15) >> 4;
     const int chunks = (p.K + 1023) >> 10;
     const uint64_t budget = p.wait_budget_ns;
+    // Without that promise B must not be READ before the previous kernel has completed -- but the L2 may be asked
+    // to fetch it: a prefetch brings no data to the SM, and the L2 stays coherent with whatever that kernel still
+    // writes.  The producer asks for the first chunks it will stream, so that its loads behind the wait start from
+    // the L2 instead of from DRAM.
+    // (Under the promise the first chunks go straight to shared memory instead; asking the L2 for the ones behind
+    // them as well only gets in the previous kernel's way: +4 to +12 % on the step.)
+    if (p.pdl_mode == 1 && !p.b_constant && warp == kRingConsumers && elect_one()) {
+        int asked = 0;
+        for (int u = blockIdx.x; u < units && asked < p.prefetch_chunks; u += gridDim.x)
+            for (int ch = 0; ch < chunks && asked < p.prefetch_chunks; ++ch, ++asked)
+                tma_prefetch_l2_3d(&p.tmap_b, 0, u * 16, ch * 8);
+    }
+    if (!(p.b_constant && warp == kRingConsumers)) pdl_wait();
+    if (warp == 0) RING_STAMP(2);
 
     if (warp == kRingConsumers) {
         // ------------------------------------------------------------ producer
